@@ -1,0 +1,156 @@
+/*
+ * flexq -- elastic mixed-bit dequantize-and-matmul for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the hot path of FlexQuant's elastic hosting scheme (arXiv 2501.07139).
+ * In that scheme a model is served from an ensemble of quantised layers and every
+ * elastic configuration ("EQM", Sec. III-A) assigns each module one of a few stored
+ * bit-widths.  This library holds the stored variants on one GPU, switches between
+ * configurations without moving weights, and runs every linear layer as a fused
+ * dequantize-and-matmul at whatever bit-width the active configuration gives it
+ * (Sec. II-A: the arithmetic itself stays in a standard 16-bit format).
+ *
+ * Conventions
+ *   - All functions return FQ_OK (0) or a negative FQ_ERR_* code.  Nothing throws,
+ *     aborts or traps.  fq_strerror() names a code.
+ *   - "dev" pointers are device memory of the context's GPU, "host" pointers are host
+ *     memory.  The library never takes ownership of a caller's buffer; buffers that a
+ *     context RETAINS must stay alive until fq_destroy().
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls on one context must be ordered on one stream (or otherwise serialised):
+ *     they share the context's workspace.
+ *   - W is [n_out][k_in] row-major, quantised per group of 128 consecutive columns:
+ *     w^ = (q - z) * s with fp16 scale s and fp16 zero point z (an integer value).
+ *     k_in must be a multiple of 128; group must be 128.
+ *   - fp16 / bf16 values cross the ABI as uint16_t bit patterns.
+ */
+#ifndef FLEXQ_H
+#define FLEXQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fq_ctx fq_ctx;   /* opaque */
+
+enum { FQ_FMT_PACKED = 0,       /* one stored variant per bit-width (Sec. III-A: QM(n) variants)   */
+       FQ_FMT_PLANES = 1 };     /* one 8-bit parent in nested bit-planes (Sec. II-B, AnyPrecision) */
+
+enum { FQ_OK = 0,
+       FQ_ERR_ARG = -1,         /* NULL pointer, bad layer index, bad enum                */
+       FQ_ERR_BITS = -2,        /* bit-width outside [2, 8] (or not 8 for a PLANES parent) */
+       FQ_ERR_SHAPE = -3,       /* group != 128, k_in % 128 != 0, sizes <= 0, batch > 8 ... */
+       FQ_ERR_ALIGN = -4,       /* a buffer is not 16-byte aligned                          */
+       FQ_ERR_NO_VARIANT = -5,  /* configuration asks for a bit-width that is not stored    */
+       FQ_ERR_NOT_PACKED = -6,  /* layer used before fq_pack_layer / fq_set_config          */
+       FQ_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, out of memory...) */
+       FQ_ERR_TIMEOUT = -8 };   /* a bounded device-side wait ran out (see fq_status)       */
+
+#define FQ_MAX_BATCH 8          /* decode batch handled by the GEMV family */
+
+/* Creates a context for `device` with room for `n_layers` layers (indices 0..n_layers-1). */
+int fq_create(fq_ctx** out, int device, int n_layers);
+/* Frees the context and its workspace.  Caller-owned buffers are not touched. */
+int fq_destroy(fq_ctx* ctx);
+
+/* Bytes the caller must allocate for the code buffer of one stored variant.  The device
+ * layout is tiled (16 rows x 256 columns), so this is the algorithmic size
+ * n_out*k_in*bits/8 (PACKED) or n_out*k_in (PLANES: the 8-bit parent) computed on
+ * n_out rounded up to 16 and k_in rounded up to 256.  Returns 0 on invalid arguments. */
+size_t fq_code_bytes(int n_out, int k_in, int bits, int fmt);
+/* Bytes for the scale/zero buffer of a layer (4 bytes per group, same rounding). */
+size_t fq_meta_bytes(int n_out, int k_in, int group);
+
+/* Min-max asymmetric group quantiser (the step in front of the path; the paper takes the
+ * quantised models QM(n) of Sec. III-A as given).  Per group of 128 columns, in double:
+ * s = fp16((max-min)/(2^b-1)) (2^-14 if that is zero), z = clamp(rint(-min/s), 0, 2^b-1),
+ * q = clamp(rint(w/s) + z, 0, 2^b-1).
+ *   w_dev      float32 [n_out][k_in]             (read)
+ *   codes_dev  uint8   [n_out][k_in], one code per byte (written)
+ *   scales_dev, zeros_dev  fp16 [n_out][k_in/128] (written)
+ * Needs no context; runs on the current device. */
+int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int group,
+                      uint8_t* codes_dev, uint16_t* scales_dev, uint16_t* zeros_dev, void* stream);
+
+/* Registers one stored variant of `layer` and converts it to the device layout
+ * (Sec. III-A: every module is stored at a few bit-widths; Sec. II-B for PLANES).
+ *   PACKED: `bits` in [2,8] is the width of this variant; call again with another width
+ *           to add a variant of the same layer (same shape).
+ *   PLANES: `bits` must be 8; the parent is stored as a 2-bit top field plus six 1-bit
+ *           planes, most significant first, so a b-bit child reads exactly the first b/8
+ *           of the buffer and every b in [2,8] becomes selectable.
+ *   codes_dev   uint8 [n_out][k_in], one code per byte; read, not retained.
+ *   scales_dev, zeros_dev   fp16 [n_out][k_in/128]; read, not retained.
+ *   code_out_dev  fq_code_bytes() bytes, 256-byte aligned; written and RETAINED.
+ *   meta_out_dev  fq_meta_bytes() bytes, 256-byte aligned; written and RETAINED.
+ * The first variant packed for a layer becomes its active one. */
+int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int group, int fmt,
+                  const uint8_t* codes_dev, const uint16_t* scales_dev, const uint16_t* zeros_dev,
+                  void* code_out_dev, void* meta_out_dev, void* stream);
+
+/* Activates an elastic configuration (Sec. III-A: an EQM is a per-module choice among the
+ * stored variants; Sec. II-C: switching should cost as little memory traffic as possible).
+ *   bits_host  uint8 [n_layers]: bit-width of every registered layer, each in [2,8].
+ *   footprint_bytes_host (may be NULL): receives the memory footprint of the configuration,
+ *       sum over layers of n_out*k_in*b/8 code bytes + n_out*(k_in/128)*4 scale/zero bytes.
+ * Fails with FQ_ERR_NO_VARIANT (and changes nothing) if a PACKED layer has no variant at
+ * the requested width.  Host-only bookkeeping: no weight byte is read, written or moved
+ * and nothing is enqueued on `stream`. */
+int fq_set_config(fq_ctx* ctx, const uint8_t* bits_host, int n_layers,
+                  uint64_t* footprint_bytes_host, void* stream);
+
+/* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
+ *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.
+ * Enqueues kernels on `stream`; does not synchronise. */
+int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
+
+/* Decode at batch 1..8:  Y[b][n] = sum_k X[b][k] * w^[n][k].
+ *   x_dev fp16 [batch][k_in], y_dev fp16 [batch][n_out], densely packed rows. */
+int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, uint16_t* y_dev, void* stream);
+
+/* Decode through a whole stack of layers in ONE persistent launch; op i computes
+ * y_dev[i] = x_dev[i] . w^(layers[i]) exactly as fq_gemv_batched would (bit-identical).
+ *   layers_host int [n_ops]; x_dev_host / y_dev_host: host arrays of n_ops device pointers.
+ *   phases_host (may be NULL = no ordering): non-decreasing int [n_ops], starting at 0 and
+ *       without gaps; an op of phase p does not read its x before every op of phase p-1 has
+ *       written its y (weights of later ops are prefetched meanwhile).
+ * May grow the context's workspace (device allocation) when the op list is larger than
+ * any seen before; otherwise enqueues one small host-to-device copy and one kernel. */
+int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host,
+                  const uint16_t* const* x_dev_host, uint16_t* const* y_dev_host,
+                  const int* phases_host, int batch, void* stream);
+
+/* Prefill / calibration-set evaluation (Sec. III-B: every candidate EQM is run forward over
+ * token sequences):  Y[m][n] = sum_k X[m][k] * w^[n][k].
+ *   X_dev bf16 [M][ldx >= k_in], Y_dev bf16 [M][ldy >= n_out], row-major, 16-byte aligned,
+ *   ldx and ldy multiples of 8.  Tensor-core path, fp32 accumulation. */
+int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx,
+            uint16_t* Y_dev, int ldy, void* stream);
+
+/* Test / reporting support ------------------------------------------------------------ */
+
+/* Writes the canonical form of what is stored for `layer` at width `bits`:
+ *   PACKED: uint32 [n_out][k_in*bits/32], per row a little-endian bitstream, code k in bits
+ *           [k*bits, (k+1)*bits).
+ *   PLANES: uint32 [bits][n_out][k_in/32], plane t holds parent bit 7-t, bit (k%32) of a
+ *           word belongs to column k; only the first `bits` stored planes are read.
+ * out_dev: n_out*k_in*bits/8 bytes. */
+int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* stream);
+/* Writes the stored scales and zero points back as fp16 [n_out][k_in/128] each. */
+int fq_export_meta(fq_ctx* ctx, int layer, int bits, uint16_t* scales_dev, uint16_t* zeros_dev, void* stream);
+
+/* Sum of the code and scale/zero bytes of every stored variant (the "storage cost" axis). */
+uint64_t fq_storage_bytes(const fq_ctx* ctx);
+/* Active bit-width of a layer, or a negative error. */
+int fq_active_bits(const fq_ctx* ctx, int layer);
+/* Synchronises the context's device, then returns and clears the device status word
+ * (FQ_OK, or FQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up). */
+int fq_status(fq_ctx* ctx);
+const char* fq_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLEXQ_H */

@@ -1,0 +1,431 @@
+// C ABI entry points: context, layer registry, configuration / footprint accountant,
+// argument checks and dispatch to the kernels.
+#include <cstring>
+#include <new>
+
+#include "fq_internal.cuh"
+
+using namespace fq;
+
+#define FQ_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return FQ_ERR_CUDA; } while (0)
+
+namespace {
+
+constexpr size_t kWsHead = 8 * 4096 + 64;      // phase counters (4096 x u64) + exit counter
+constexpr int kMaxPhases = 4096;
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = prev == dev || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+FieldList active_fields(const Layer& L, int bits) { return L.fmt == FQ_FMT_PLANES ? plane_fields(bits) : packed_fields(bits); }
+
+const Variant* active_variant(const Layer& L, int bits)
+{
+    const Variant& v = L.fmt == FQ_FMT_PLANES ? L.var[8] : L.var[bits];
+    return v.present ? &v : nullptr;
+}
+
+// Fills the device descriptor of one decode op (everything except workspace pointers and unit_base).
+int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch, GemvOp& op)
+{
+    if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    const Layer& L = ctx->layers[layer];
+    if (!L.registered || L.active_bits == 0) return FQ_ERR_NOT_PACKED;
+    if (!x || !y) return FQ_ERR_ARG;
+    if (batch < 1 || batch > FQ_MAX_BATCH) return FQ_ERR_SHAPE;
+    if (!aligned(x, 16) || !aligned(y, 16)) return FQ_ERR_ALIGN;
+    const int bits = L.active_bits;
+    const Variant* v = active_variant(L, bits);
+    if (!v) return FQ_ERR_NO_VARIANT;
+    const FieldList fl = active_fields(L, bits);
+    std::memset(&op, 0, sizeof op);
+    const uint8_t* p = static_cast<const uint8_t*>(v->codes);
+    for (int i = 0; i < fl.n; i++) {
+        op.field_ptr[i] = p;
+        op.field_width[i] = fl.width[i];
+        op.field_shift[i] = fl.shift[i];
+        p += field_bytes(L.n_out, L.k_in, fl.width[i]);
+    }
+    op.n_fields = fl.n;
+    op.bits = bits;
+    op.meta = static_cast<const uint32_t*>(v->meta);
+    op.x = x;
+    op.y = y;
+    op.n_out = L.n_out;
+    op.k_in = L.k_in;
+    op.n_rt = row_tiles(L.n_out);
+    op.n_ss = supersteps(L.k_in);
+    op.n_chunks = gemv_chunks(op.n_ss, bits, batch);
+    op.batch = batch;
+    // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
+    op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (float)(1 << (7 - bits)) : 0.f;
+    op.phase = -1;
+    op.unit_base = 0;
+    return FQ_OK;
+}
+
+size_t op_partial_bytes(const GemvOp& op, int max_batch)
+{
+    if (op.n_chunks <= 1) return 0;
+    return (size_t)op.n_rt * op.n_chunks * gemv_partial_floats_per_unit(max_batch) * sizeof(float);
+}
+size_t op_counter_bytes(const GemvOp& op) { return op.n_chunks <= 1 ? 0 : (size_t)round_up(op.n_rt * 4, 16); }
+
+uint64_t hash_mix(uint64_t h, uint64_t v)
+{
+    h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
+    return h;
+}
+
+}  // namespace
+
+namespace fq {
+
+int ensure_workspace(Ctx* ctx, size_t bytes)
+{
+    if (bytes <= ctx->ws_bytes) return FQ_OK;
+    const size_t want = (size_t)round_up((int64_t)(bytes + bytes / 4), 1 << 20);
+    char* p = nullptr;
+    FQ_CUDA_OK(cudaDeviceSynchronize());
+    FQ_CUDA_OK(cudaMalloc(&p, want));
+    if (cudaMemset(p, 0, want) != cudaSuccess) { cudaFree(p); return FQ_ERR_CUDA; }
+    FQ_CUDA_OK(cudaDeviceSynchronize());
+    if (ctx->ws) cudaFree(ctx->ws);
+    ctx->ws = p;
+    ctx->ws_bytes = want;
+    ctx->stack_valid = false;          // cached op tables point into the old workspace
+    return FQ_OK;
+}
+
+}  // namespace fq
+
+extern "C" {
+
+const char* fq_strerror(int code)
+{
+    switch (code) {
+        case FQ_OK: return "ok";
+        case FQ_ERR_ARG: return "invalid argument";
+        case FQ_ERR_BITS: return "bit-width out of range";
+        case FQ_ERR_SHAPE: return "unsupported shape";
+        case FQ_ERR_ALIGN: return "buffer not aligned";
+        case FQ_ERR_NO_VARIANT: return "no stored variant at this bit-width";
+        case FQ_ERR_NOT_PACKED: return "layer not packed";
+        case FQ_ERR_CUDA: return "CUDA runtime error";
+        case FQ_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown error";
+    }
+}
+
+int fq_create(fq_ctx** out, int device, int n_layers)
+{
+    if (!out || n_layers < 1 || n_layers > (1 << 20) || device < 0) return FQ_ERR_ARG;
+    *out = nullptr;
+    int count = 0;
+    FQ_CUDA_OK(cudaGetDeviceCount(&count));
+    if (device >= count) return FQ_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    fq_ctx* ctx = new (std::nothrow) fq_ctx();
+    if (!ctx) return FQ_ERR_ARG;
+    ctx->device = device;
+    ctx->layers.resize(n_layers);
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaMalloc(&ctx->status_dev, sizeof(int)) != cudaSuccess ||
+        cudaMemset(ctx->status_dev, 0, sizeof(int)) != cudaSuccess ||
+        ensure_workspace(ctx, kWsHead + (1 << 20)) != FQ_OK) {
+        if (ctx->status_dev) cudaFree(ctx->status_dev);
+        delete ctx;
+        return FQ_ERR_CUDA;
+    }
+    *out = ctx;
+    return FQ_OK;
+}
+
+int fq_destroy(fq_ctx* ctx)
+{
+    if (!ctx) return FQ_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (guard.ok) {
+        cudaDeviceSynchronize();
+        if (ctx->ws) cudaFree(ctx->ws);
+        if (ctx->status_dev) cudaFree(ctx->status_dev);
+        if (ctx->stack_dev) cudaFree(ctx->stack_dev);
+        if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
+    }
+    delete ctx;
+    return FQ_OK;
+}
+
+size_t fq_code_bytes(int n_out, int k_in, int bits, int fmt)
+{
+    if (n_out < 1 || k_in < 1 || k_in % kGroup != 0) return 0;
+    if (fmt == FQ_FMT_PLANES) { if (bits != 8) return 0; }
+    else if (fmt == FQ_FMT_PACKED) { if (bits < 2 || bits > 8) return 0; }
+    else return 0;
+    return (size_t)row_tiles(n_out) * supersteps(k_in) * 512 * bits;
+}
+
+size_t fq_meta_bytes(int n_out, int k_in, int group)
+{
+    if (n_out < 1 || k_in < 1 || group != kGroup || k_in % kGroup != 0) return 0;
+    return (size_t)row_tiles(n_out) * supersteps(k_in) * 2 * 16 * 4;
+}
+
+int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int group,
+                      uint8_t* codes_dev, uint16_t* scales_dev, uint16_t* zeros_dev, void* stream)
+{
+    if (!w_dev || !codes_dev || !scales_dev || !zeros_dev) return FQ_ERR_ARG;
+    if (bits < 2 || bits > 8) return FQ_ERR_BITS;
+    if (group != kGroup || n_out < 1 || k_in < 1 || k_in % kGroup != 0) return FQ_ERR_SHAPE;
+    if (!aligned(w_dev, 16) || !aligned(codes_dev, 4)) return FQ_ERR_ALIGN;
+    return launch_quantize(w_dev, n_out, k_in, bits, codes_dev, scales_dev, zeros_dev, (cudaStream_t)stream);
+}
+
+int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int group, int fmt,
+                  const uint8_t* codes_dev, const uint16_t* scales_dev, const uint16_t* zeros_dev,
+                  void* code_out_dev, void* meta_out_dev, void* stream)
+{
+    if (!ctx || !codes_dev || !scales_dev || !zeros_dev || !code_out_dev || !meta_out_dev) return FQ_ERR_ARG;
+    if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    if (fmt != FQ_FMT_PACKED && fmt != FQ_FMT_PLANES) return FQ_ERR_ARG;
+    if (bits < 2 || bits > 8 || (fmt == FQ_FMT_PLANES && bits != 8)) return FQ_ERR_BITS;
+    if (group != kGroup || n_out < 1 || k_in < 1 || k_in % kGroup != 0) return FQ_ERR_SHAPE;
+    if (!aligned(code_out_dev, 256) || !aligned(meta_out_dev, 256)) return FQ_ERR_ALIGN;
+    Layer& L = ctx->layers[layer];
+    if (L.registered && (L.n_out != n_out || L.k_in != k_in || L.fmt != fmt)) return FQ_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    const FieldList fl = fmt == FQ_FMT_PLANES ? plane_fields(8) : packed_fields(bits);
+    const int rc = launch_pack(codes_dev, scales_dev, zeros_dev, n_out, k_in, fl, code_out_dev, meta_out_dev,
+                               (cudaStream_t)stream);
+    if (rc != FQ_OK) return rc;
+    L.registered = true;
+    L.n_out = n_out; L.k_in = k_in; L.fmt = fmt;
+    Variant& v = L.var[bits];
+    v.present = true; v.codes = code_out_dev; v.meta = meta_out_dev;
+    if (L.active_bits == 0) L.active_bits = bits;
+    ctx->config_epoch++;
+    return FQ_OK;
+}
+
+int fq_set_config(fq_ctx* ctx, const uint8_t* bits_host, int n_layers, uint64_t* footprint_bytes_host, void* stream)
+{
+    (void)stream;
+    if (!ctx || !bits_host) return FQ_ERR_ARG;
+    int registered = 0;
+    for (const Layer& L : ctx->layers) registered += L.registered ? 1 : 0;
+    if (n_layers != registered) return FQ_ERR_ARG;
+    // validate everything first so a failing call changes nothing
+    uint64_t total = 0;
+    int i = 0;
+    for (const Layer& L : ctx->layers) {
+        if (!L.registered) continue;
+        const int b = bits_host[i++];
+        if (b < 2 || b > 8) return FQ_ERR_BITS;
+        if (!active_variant(L, b)) return FQ_ERR_NO_VARIANT;
+        total += (uint64_t)L.n_out * (uint64_t)L.k_in * (uint64_t)b / 8u;
+        total += (uint64_t)L.n_out * (uint64_t)(L.k_in / kGroup) * 4u;
+    }
+    i = 0;
+    for (Layer& L : ctx->layers)
+        if (L.registered) L.active_bits = bits_host[i++];
+    ctx->config_epoch++;
+    if (footprint_bytes_host) *footprint_bytes_host = total;
+    return FQ_OK;
+}
+
+uint64_t fq_storage_bytes(const fq_ctx* ctx)
+{
+    if (!ctx) return 0;
+    uint64_t total = 0;
+    for (const Layer& L : ctx->layers) {
+        if (!L.registered) continue;
+        const uint64_t meta = (uint64_t)L.n_out * (uint64_t)(L.k_in / kGroup) * 4u;
+        for (int b = 2; b <= 8; b++)
+            if (L.var[b].present) total += (uint64_t)L.n_out * (uint64_t)L.k_in * (uint64_t)b / 8u + meta;
+    }
+    return total;
+}
+
+int fq_active_bits(const fq_ctx* ctx, int layer)
+{
+    if (!ctx || layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    const Layer& L = ctx->layers[layer];
+    if (!L.registered) return FQ_ERR_NOT_PACKED;
+    return L.active_bits;
+}
+
+int fq_status(fq_ctx* ctx)
+{
+    if (!ctx) return FQ_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    FQ_CUDA_OK(cudaDeviceSynchronize());
+    int st = 0;
+    FQ_CUDA_OK(cudaMemcpy(&st, ctx->status_dev, sizeof st, cudaMemcpyDeviceToHost));
+    if (st != 0) {
+        // counters may have been left half-way: start from a clean workspace
+        FQ_CUDA_OK(cudaMemset(ctx->status_dev, 0, sizeof(int)));
+        FQ_CUDA_OK(cudaMemset(ctx->ws, 0, ctx->ws_bytes));
+        FQ_CUDA_OK(cudaDeviceSynchronize());
+    }
+    return st;
+}
+
+int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, uint16_t* y_dev, void* stream)
+{
+    if (!ctx) return FQ_ERR_ARG;
+    GemvOp op;
+    int rc = fill_op(ctx, layer, x_dev, y_dev, batch, op);
+    if (rc != FQ_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    const size_t pb = op_partial_bytes(op, batch), cb = op_counter_bytes(op);
+    rc = ensure_workspace(ctx, kWsHead + cb + pb + 256);
+    if (rc != FQ_OK) return rc;
+    op.tile_count = reinterpret_cast<unsigned*>(ctx->ws + kWsHead);
+    op.partial = reinterpret_cast<float*>(ctx->ws + kWsHead + round_up((int64_t)cb, 256));
+    return launch_gemv_single(ctx, op, (cudaStream_t)stream);
+}
+
+int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream)
+{
+    return fq_gemv_batched(ctx, layer, x_dev, 1, y_dev, stream);
+}
+
+int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t* const* x_dev_host,
+                  uint16_t* const* y_dev_host, const int* phases_host, int batch, void* stream)
+{
+    if (!ctx || !layers_host || !x_dev_host || !y_dev_host || n_ops < 1) return FQ_ERR_ARG;
+    if (batch < 1 || batch > FQ_MAX_BATCH) return FQ_ERR_SHAPE;
+    int n_phases = 0;
+    if (phases_host) {
+        if (phases_host[0] != 0) return FQ_ERR_ARG;
+        for (int i = 1; i < n_ops; i++)
+            if (phases_host[i] < phases_host[i - 1] || phases_host[i] > phases_host[i - 1] + 1) return FQ_ERR_ARG;
+        n_phases = phases_host[n_ops - 1] + 1;
+        if (n_phases > kMaxPhases) return FQ_ERR_SHAPE;
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+
+    // The op table only depends on the arguments and the active configuration: reuse the
+    // uploaded copy when neither changed.
+    uint64_t key = hash_mix(0x51ed27, (uint64_t)n_ops);
+    key = hash_mix(key, ctx->config_epoch);
+    key = hash_mix(key, (uint64_t)batch);
+    for (int i = 0; i < n_ops; i++) {
+        key = hash_mix(key, (uint64_t)layers_host[i]);
+        key = hash_mix(key, (uint64_t)reinterpret_cast<uintptr_t>(x_dev_host[i]));
+        key = hash_mix(key, (uint64_t)reinterpret_cast<uintptr_t>(y_dev_host[i]));
+        key = hash_mix(key, phases_host ? (uint64_t)phases_host[i] : ~0ull);
+    }
+    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) + (size_t)(n_phases > 0 ? n_phases : 1) * sizeof(long long);
+    const size_t hdr_off = (size_t)round_up((int64_t)table_bytes, 16);
+    StackHeader hdr{};
+
+    if (!(ctx->stack_valid && ctx->stack_key == key)) {
+        if (ctx->stack_host_bytes < hdr_off + sizeof(StackHeader)) {
+            if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
+            ctx->stack_host = nullptr; ctx->stack_host_bytes = 0;
+            const size_t want = 2 * (hdr_off + sizeof(StackHeader));
+            FQ_CUDA_OK(cudaMallocHost(&ctx->stack_host, want));
+            ctx->stack_host_bytes = want;
+        }
+        GemvOp* ops = reinterpret_cast<GemvOp*>(ctx->stack_host);
+        long long* phase_total = reinterpret_cast<long long*>(ctx->stack_host + (size_t)n_ops * sizeof(GemvOp));
+        for (int p = 0; p < (n_phases > 0 ? n_phases : 1); p++) phase_total[p] = 0;
+        size_t ws_need = kWsHead;
+        long long unit_base = 0;
+        for (int i = 0; i < n_ops; i++) {
+            const int rc = fill_op(ctx, layers_host[i], x_dev_host[i], y_dev_host[i], batch, ops[i]);
+            if (rc != FQ_OK) return rc;
+            ops[i].phase = phases_host ? phases_host[i] : -1;
+            ops[i].unit_base = unit_base;
+            const long long units = (long long)ops[i].n_rt * ops[i].n_chunks;
+            unit_base += units;
+            if (phases_host) phase_total[phases_host[i]] += units;
+            ws_need = (size_t)round_up((int64_t)ws_need, 256);
+            ws_need += op_counter_bytes(ops[i]);
+            ws_need = (size_t)round_up((int64_t)ws_need, 256);
+            ws_need += op_partial_bytes(ops[i], batch);
+        }
+        int rc = ensure_workspace(ctx, ws_need + 256);
+        if (rc != FQ_OK) return rc;
+        size_t off = kWsHead;
+        for (int i = 0; i < n_ops; i++) {
+            off = (size_t)round_up((int64_t)off, 256);
+            ops[i].tile_count = reinterpret_cast<unsigned*>(ctx->ws + off);
+            off += op_counter_bytes(ops[i]);
+            off = (size_t)round_up((int64_t)off, 256);
+            ops[i].partial = reinterpret_cast<float*>(ctx->ws + off);
+            off += op_partial_bytes(ops[i], batch);
+        }
+        hdr.n_ops = n_ops; hdr.n_phases = n_phases; hdr.total_units = unit_base;
+        std::memcpy(ctx->stack_host + hdr_off, &hdr, sizeof hdr);
+        if (ctx->stack_dev_bytes < table_bytes) {
+            FQ_CUDA_OK(cudaDeviceSynchronize());
+            if (ctx->stack_dev) cudaFree(ctx->stack_dev);
+            ctx->stack_dev = nullptr; ctx->stack_dev_bytes = 0;
+            FQ_CUDA_OK(cudaMalloc(&ctx->stack_dev, 2 * table_bytes));
+            ctx->stack_dev_bytes = 2 * table_bytes;
+        }
+        FQ_CUDA_OK(cudaMemcpyAsync(ctx->stack_dev, ctx->stack_host, table_bytes, cudaMemcpyHostToDevice,
+                                   (cudaStream_t)stream));
+        ctx->stack_key = key;
+        ctx->stack_valid = true;
+    } else {
+        std::memcpy(&hdr, ctx->stack_host + hdr_off, sizeof hdr);
+    }
+    return launch_gemv_stack(ctx, hdr, ctx->stack_dev, batch, (cudaStream_t)stream);
+}
+
+int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)
+{
+    (void)ctx; (void)layer; (void)X_dev; (void)M; (void)ldx; (void)Y_dev; (void)ldy; (void)stream;
+    return FQ_ERR_ARG;
+}
+
+int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* stream)
+{
+    if (!ctx || !out_dev || layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    if (bits < 2 || bits > 8) return FQ_ERR_BITS;
+    const Layer& L = ctx->layers[layer];
+    if (!L.registered) return FQ_ERR_NOT_PACKED;
+    const Variant* v = active_variant(L, bits);
+    if (!v) return FQ_ERR_NO_VARIANT;
+    if (!aligned(out_dev, 4)) return FQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    if (L.fmt == FQ_FMT_PLANES)
+        return launch_export_planes(v->codes, L.n_out, L.k_in, bits, plane_fields(bits), (uint32_t*)out_dev,
+                                    (cudaStream_t)stream);
+    return launch_export_packed(v->codes, L.n_out, L.k_in, bits, packed_fields(bits), (uint32_t*)out_dev,
+                                (cudaStream_t)stream);
+}
+
+int fq_export_meta(fq_ctx* ctx, int layer, int bits, uint16_t* scales_dev, uint16_t* zeros_dev, void* stream)
+{
+    if (!ctx || !scales_dev || !zeros_dev || layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    if (bits < 2 || bits > 8) return FQ_ERR_BITS;
+    const Layer& L = ctx->layers[layer];
+    if (!L.registered) return FQ_ERR_NOT_PACKED;
+    const Variant* v = active_variant(L, bits);
+    if (!v) return FQ_ERR_NO_VARIANT;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    return launch_export_meta(v->meta, L.n_out, L.k_in, scales_dev, zeros_dev, (cudaStream_t)stream);
+}
+
+}  // extern "C"

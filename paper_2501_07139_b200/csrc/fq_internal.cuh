@@ -1,0 +1,93 @@
+// Host-side context and the descriptors passed to the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <vector>
+
+#include "../../include/flexq.h"
+#include "fq_layout.cuh"
+
+namespace fq {
+
+// One stored variant of a layer.
+struct Variant {
+    bool present = false;
+    void* codes = nullptr;       // field arrays, concatenated, most significant first
+    void* meta = nullptr;        // [row_tile][group][16] (scale, zero) words
+};
+
+struct Layer {
+    bool registered = false;
+    int n_out = 0, k_in = 0, fmt = FQ_FMT_PACKED;
+    int active_bits = 0;
+    Variant var[9];              // PACKED: index = bits; PLANES: only [8]
+};
+
+// What one decode op needs on the device.
+struct GemvOp {
+    const uint8_t* field_ptr[kMaxFields];
+    uint8_t field_width[kMaxFields];
+    uint8_t field_shift[kMaxFields];
+    int n_fields;
+    int bits;                    // code bytes per tile superstep = 512 * bits
+    const uint32_t* meta;
+    const uint16_t* x;           // fp16 [batch][k_in]
+    uint16_t* y;                 // fp16 [batch][n_out]
+    float* partial;              // split-K partial sums (unused when n_chunks == 1)
+    unsigned* tile_count;        // split-K arrival counters, one per row tile
+    int n_out, k_in;
+    int n_rt, n_ss;              // row tiles, supersteps
+    int n_chunks;                // K chunks per row tile
+    int batch;
+    float zero_adjust;           // subtracted from every zero point (mid-point fill of a nested child)
+    int phase;                   // -1: no ordering
+    long long unit_base;         // global index of this op's first unit
+};
+
+struct StackHeader {
+    int n_ops;
+    int n_phases;
+    long long total_units;
+};
+
+struct Ctx {
+    int device = 0;
+    int sm_count = 0;
+    std::vector<Layer> layers;
+    // workspace shared by all calls on this context
+    char* ws = nullptr;          // device
+    size_t ws_bytes = 0;
+    int* status_dev = nullptr;   // device status word
+    // stack-call staging
+    char* stack_dev = nullptr;   // device copy of the op table
+    size_t stack_dev_bytes = 0;
+    char* stack_host = nullptr;  // pinned
+    size_t stack_host_bytes = 0;
+    uint64_t config_epoch = 0;
+    uint64_t stack_key = 0;      // hash of the op list that is currently uploaded
+    bool stack_valid = false;
+};
+
+// Bytes of device workspace for `n_ops` ops whose split-K needs are summed by the caller.
+int ensure_workspace(Ctx* ctx, size_t bytes);
+
+// kernels / launchers implemented in the .cu files
+int launch_quantize(const float* w, int n_out, int k_in, int bits, uint8_t* codes, uint16_t* scales,
+                    uint16_t* zeros, cudaStream_t st);
+int launch_pack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int n_out, int k_in,
+                const FieldList& fl, void* code_out, void* meta_out, cudaStream_t st);
+int launch_export_packed(const void* codes, int n_out, int k_in, int bits, const FieldList& fl,
+                         uint32_t* out, cudaStream_t st);
+int launch_export_planes(const void* codes, int n_out, int k_in, int bits, const FieldList& fl,
+                         uint32_t* out, cudaStream_t st);
+int launch_export_meta(const void* meta, int n_out, int k_in, uint16_t* scales, uint16_t* zeros, cudaStream_t st);
+
+// Chunking policy of the decode kernel: number of K chunks per row tile.
+int gemv_chunks(int n_ss, int bits, int batch);
+size_t gemv_partial_floats_per_unit(int batch);
+int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
+int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
+
+}  // namespace fq
+
+struct fq_ctx : fq::Ctx {};

@@ -1,0 +1,226 @@
+"""ctypes binding of libflexq.so: argument marshalling only.
+
+Every method has the name of the C function it calls.  torch is used for device memory
+and streams; all computation happens inside the library's CUDA kernels.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+FQ_FMT_PACKED = 0
+FQ_FMT_PLANES = 1
+FQ_MAX_BATCH = 8
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libflexq.so")
+_lib = None
+
+EXPORTS = [
+    "fq_create", "fq_destroy", "fq_code_bytes", "fq_meta_bytes", "fq_quantize_layer", "fq_pack_layer",
+    "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
+    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror",
+]
+
+
+class FlexQError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {fq_strerror(code)} ({code})")
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """Loads libflexq.so (once).  Raises if it is missing: build it with
+    `python -m paper_2501_07139_b200.build` or `__graft_entry__.build()`."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise FileNotFoundError(f"{_LIB_PATH} not built; run `python -m paper_2501_07139_b200.build`")
+    L = C.CDLL(_LIB_PATH)
+    vp, i, u64 = C.c_void_p, C.c_int, C.c_uint64
+    L.fq_create.argtypes = [C.POINTER(vp), i, i]
+    L.fq_destroy.argtypes = [vp]
+    L.fq_code_bytes.argtypes = [i, i, i, i]
+    L.fq_code_bytes.restype = C.c_size_t
+    L.fq_meta_bytes.argtypes = [i, i, i]
+    L.fq_meta_bytes.restype = C.c_size_t
+    L.fq_quantize_layer.argtypes = [vp, i, i, i, i, vp, vp, vp, vp]
+    L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp]
+    L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
+    L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
+    L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
+    L.fq_gemv_stack.argtypes = [vp, i, vp, vp, vp, vp, i, vp]
+    L.fq_gemm.argtypes = [vp, i, vp, i, i, vp, i, vp]
+    L.fq_export_layer.argtypes = [vp, i, i, vp, vp]
+    L.fq_export_meta.argtypes = [vp, i, i, vp, vp, vp]
+    L.fq_storage_bytes.argtypes = [vp]
+    L.fq_storage_bytes.restype = u64
+    L.fq_active_bits.argtypes = [vp, i]
+    L.fq_status.argtypes = [vp]
+    L.fq_strerror.argtypes = [i]
+    L.fq_strerror.restype = C.c_char_p
+    for name in EXPORTS:
+        fn = getattr(L, name)
+        if fn.restype is C.c_int or fn.restype is None:
+            fn.restype = C.c_int
+    _lib = L
+    return L
+
+
+def fq_strerror(code: int) -> str:
+    return lib().fq_strerror(int(code)).decode()
+
+
+def fq_code_bytes(n_out: int, k_in: int, bits: int, fmt: int) -> int:
+    return int(lib().fq_code_bytes(n_out, k_in, bits, fmt))
+
+
+def fq_meta_bytes(n_out: int, k_in: int, group: int = 128) -> int:
+    return int(lib().fq_meta_bytes(n_out, k_in, group))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc: int, where: str) -> int:
+    if rc != 0:
+        raise FlexQError(rc, where)
+    return rc
+
+
+def fq_quantize_layer(w: torch.Tensor, bits: int, group: int = 128):
+    """W float32 [N][K] on the GPU -> (codes uint8 [N][K], scales fp16 [N][K/128], zeros fp16 [N][K/128])."""
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+    n, k = w.shape
+    codes = torch.empty((n, k), dtype=torch.uint8, device=w.device)
+    scales = torch.empty((n, k // group), dtype=torch.float16, device=w.device)
+    zeros = torch.empty((n, k // group), dtype=torch.float16, device=w.device)
+    with torch.cuda.device(w.device):
+        _check(lib().fq_quantize_layer(w.data_ptr(), n, k, bits, group, codes.data_ptr(), scales.data_ptr(),
+                                       zeros.data_ptr(), _stream()), "fq_quantize_layer")
+    return codes, scales, zeros
+
+
+class FlexQ:
+    """One library context.  Keeps the retained device buffers (codes, metadata) alive."""
+
+    def __init__(self, n_layers: int, device: int = 0):
+        self._h = C.c_void_p()
+        self.device = torch.device("cuda", device)
+        _check(lib().fq_create(C.byref(self._h), device, n_layers), "fq_create")
+        self.n_layers = n_layers
+        self._keep = {}          # (layer, bits) -> (codes, meta) tensors retained by the context
+        self._stack_keep = None
+
+    # -- lifetime -----------------------------------------------------------------
+    def fq_destroy(self):
+        if self._h:
+            lib().fq_destroy(self._h)
+            self._h = C.c_void_p()
+            self._keep.clear()
+
+    def __del__(self):
+        try:
+            self.fq_destroy()
+        except Exception:
+            pass
+
+    # -- packing --------------------------------------------------------------------
+    def fq_pack_layer(self, layer: int, codes: torch.Tensor, scales: torch.Tensor, zeros: torch.Tensor,
+                      bits: int, fmt: int = FQ_FMT_PACKED, group: int = 128):
+        assert codes.is_cuda and codes.dtype == torch.uint8 and codes.is_contiguous()
+        assert scales.dtype == torch.float16 and zeros.dtype == torch.float16
+        n, k = codes.shape
+        cb, mb = fq_code_bytes(n, k, bits, fmt), fq_meta_bytes(n, k, group)
+        if cb == 0 or mb == 0:
+            # let the library name the problem
+            _check(lib().fq_pack_layer(self._h, layer, n, k, bits, group, fmt, codes.data_ptr(), scales.data_ptr(),
+                                       zeros.data_ptr(), codes.data_ptr(), codes.data_ptr(), _stream()),
+                   "fq_pack_layer")
+        code_out = torch.empty(cb, dtype=torch.uint8, device=self.device)
+        meta_out = torch.empty(mb, dtype=torch.uint8, device=self.device)
+        _check(lib().fq_pack_layer(self._h, layer, n, k, bits, group, fmt, codes.data_ptr(),
+                                   scales.contiguous().data_ptr(), zeros.contiguous().data_ptr(),
+                                   code_out.data_ptr(), meta_out.data_ptr(), _stream()), "fq_pack_layer")
+        self._keep[(layer, bits)] = (code_out, meta_out)
+        return code_out, meta_out
+
+    # -- configuration -------------------------------------------------------------------
+    def fq_set_config(self, bits: Sequence[int]) -> int:
+        arr = (C.c_uint8 * len(bits))(*[int(b) for b in bits])
+        fp = C.c_uint64(0)
+        _check(lib().fq_set_config(self._h, arr, len(bits), C.byref(fp), _stream()), "fq_set_config")
+        return int(fp.value)
+
+    def fq_storage_bytes(self) -> int:
+        return int(lib().fq_storage_bytes(self._h))
+
+    def fq_active_bits(self, layer: int) -> int:
+        rc = lib().fq_active_bits(self._h, layer)
+        if rc < 0:
+            raise FlexQError(rc, "fq_active_bits")
+        return rc
+
+    def fq_status(self) -> int:
+        return int(lib().fq_status(self._h))
+
+    # -- decode --------------------------------------------------------------------------
+    def fq_gemv(self, layer: int, x: torch.Tensor, y: torch.Tensor):
+        _check(lib().fq_gemv(self._h, layer, x.data_ptr(), y.data_ptr(), _stream()), "fq_gemv")
+        return y
+
+    def fq_gemv_batched(self, layer: int, x: torch.Tensor, y: torch.Tensor):
+        _check(lib().fq_gemv_batched(self._h, layer, x.data_ptr(), x.shape[0], y.data_ptr(), _stream()),
+               "fq_gemv_batched")
+        return y
+
+    def fq_gemv_stack(self, layers: Sequence[int], xs: Sequence[torch.Tensor], ys: Sequence[torch.Tensor],
+                      phases: Optional[Sequence[int]] = None, batch: int = 1):
+        n = len(layers)
+        la = (C.c_int * n)(*[int(v) for v in layers])
+        xa = (C.c_void_p * n)(*[t.data_ptr() for t in xs])
+        ya = (C.c_void_p * n)(*[t.data_ptr() for t in ys])
+        pa = (C.c_int * n)(*[int(v) for v in phases]) if phases is not None else None
+        self._stack_keep = (la, xa, ya, pa)
+        _check(lib().fq_gemv_stack(self._h, n, la, xa, ya, pa, batch, _stream()), "fq_gemv_stack")
+
+    def stack_args(self, layers, xs, ys, phases=None):
+        """Pre-marshalled argument arrays for repeated fq_gemv_stack_raw calls."""
+        n = len(layers)
+        la = (C.c_int * n)(*[int(v) for v in layers])
+        xa = (C.c_void_p * n)(*[t.data_ptr() for t in xs])
+        ya = (C.c_void_p * n)(*[t.data_ptr() for t in ys])
+        pa = (C.c_int * n)(*[int(v) for v in phases]) if phases is not None else None
+        return (n, la, xa, ya, pa)
+
+    def fq_gemv_stack_raw(self, args, batch: int = 1):
+        n, la, xa, ya, pa = args
+        _check(lib().fq_gemv_stack(self._h, n, la, xa, ya, pa, batch, _stream()), "fq_gemv_stack")
+
+    # -- prefill --------------------------------------------------------------------------
+    def fq_gemm(self, layer: int, X: torch.Tensor, Y: torch.Tensor):
+        assert X.dtype == torch.bfloat16 and Y.dtype == torch.bfloat16
+        _check(lib().fq_gemm(self._h, layer, X.data_ptr(), X.shape[0], X.stride(0), Y.data_ptr(), Y.stride(0),
+                             _stream()), "fq_gemm")
+        return Y
+
+    # -- export (tests / reporting) ----------------------------------------------------------
+    def fq_export_layer(self, layer: int, bits: int, n_out: int, k_in: int) -> torch.Tensor:
+        out = torch.empty(n_out * k_in * bits // 32, dtype=torch.int32, device=self.device)
+        _check(lib().fq_export_layer(self._h, layer, bits, out.data_ptr(), _stream()), "fq_export_layer")
+        return out
+
+    def fq_export_meta(self, layer: int, bits: int, n_out: int, k_in: int):
+        s = torch.empty((n_out, k_in // 128), dtype=torch.float16, device=self.device)
+        z = torch.empty((n_out, k_in // 128), dtype=torch.float16, device=self.device)
+        _check(lib().fq_export_meta(self._h, layer, bits, s.data_ptr(), z.data_ptr(), _stream()), "fq_export_meta")
+        return s, z
