@@ -1,0 +1,318 @@
+#!/usr/bin/env python
+"""Benchmark of the elastic mixed-bit decode path on B200.
+
+One "step" is one pass of the hot path over the Llama-2-7B-shaped layer stack: a batch-1
+fp16 activation vector goes through all 224 packed mixed-bit matrices (bits per matrix drawn
+from {3,4,5,6,8}, group 128) in ONE persistent fq_gemv_stack launch that honours the
+dependency order {q,k,v} -> o -> {gate,up} -> down -> next block.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--blocks B]
+
+Prints one JSON line (rank 0).  N > 1 runs N independent replicas (the path does not shard).
+`--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import fq_synth as S
+
+METRIC = "mixed-bit dequant-GEMV weight GB/s"
+UNIT = "GB/s"
+CONFIG_ID = 1                      # the 7B decode stack
+BIT_CHOICES = [3, 4, 5, 6, 8]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+def read_ncu_traffic(footprint_bytes):
+    """DRAM bytes per stack launch derived from the committed ncu capture of a small case
+    (traffic / algorithmic bytes there, times this launch's algorithmic bytes).  None when the
+    kernel source changed after the counters were taken."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "gemv_stack_traffic.json")) as f:
+            d = json.load(f)
+        with open(os.path.join(ROOT, "paper_2501_07139_b200", "csrc", "fq_gemv.cu"), "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+        if sha != d["source_sha256"]:
+            return None, "kernel changed since the ncu capture"
+        return d["ratio"] * footprint_bytes, d["note"]
+    except Exception:
+        return None, "no ncu capture recorded"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            p = [c.strip() for c in r.split(",")]
+            if len(p) < 6:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_stack(P, shapes, bits, device):
+    """Seeded weights -> GPU quantiser -> packed layers.  Returns the context."""
+    fq = P.FlexQ(len(shapes), device.index or 0)
+    for i, (sh, b) in enumerate(zip(shapes, bits)):
+        w = S.weight_rows(S.tensor_key(CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device)
+        c, s, z = P.fq_quantize_layer(w, int(b))
+        fq.fq_pack_layer(i, c, s, z, int(b), P.FQ_FMT_PACKED)
+        del w, c, s, z
+    torch.cuda.synchronize()
+    return fq
+
+
+def oracle_sample(shapes, bits, n_layers, device_for_gen):
+    """Times the CPU oracle's GEMV on the first `n_layers` matrices of the workload.
+    Returns (bytes processed, seconds, description)."""
+    from oracle import fq_oracle as O
+    O.build()
+    total_bytes, total_s = 0, 0.0
+    for i in range(n_layers):
+        sh, b = shapes[i], int(bits[i])
+        w = S.weight_rows(S.tensor_key(CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device_for_gen)
+        codes, sc, zr = O.quantize(w.cpu().numpy(), b)
+        x = S.activations(S.tensor_key(CONFIG_ID, i, S.TENSOR_X), 1, sh.k_in, torch.float16)
+        xb = x.view(torch.int16).numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        O.gemv(codes, sc, zr, b, xb)
+        total_s += time.perf_counter() - t0
+        total_bytes += sh.n_out * sh.k_in * b // 8 + sh.n_out * (sh.k_in // 128) * 4
+    return total_bytes, total_s, f"oracle GEMV over the first {n_layers} matrices (block 0) of the stack, single thread"
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    shapes = S.stack_shapes("7b", args.blocks)
+    bits = S.draw_bits(S.tensor_key(CONFIG_ID, 0, S.TENSOR_BITS), len(shapes), BIT_CHOICES)
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    n_layers = min(args.ref_layers, len(shapes))
+    times, byts = [], 0
+    for step in range(args.warmup + args.steps):
+        byts, secs, desc = oracle_sample(shapes, bits, n_layers, gen_dev)
+        if step >= args.warmup:
+            times.append(secs)
+    t = float(np.mean(times))
+    val = byts / t / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"llama2-7b-shaped decode stack, {len(shapes)} matrices, bits {BIT_CHOICES}, g=128, batch 1",
+                   "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--blocks", type=int, default=32, help="decoder blocks of the 7B-shaped stack (32 = full)")
+    ap.add_argument("--ref-layers", type=int, default=7, help="matrices the CPU oracle is timed on")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+
+    import paper_2501_07139_b200 as P
+    P.lib()                                      # fails loudly if the CUDA library is missing
+
+    shapes = S.stack_shapes("7b", args.blocks)
+    L = len(shapes)
+    bits = S.draw_bits(S.tensor_key(CONFIG_ID, 0, S.TENSOR_BITS), L, BIT_CHOICES)
+    phases = S.stack_phases(shapes)
+    fq = build_stack(P, shapes, bits, device)
+    footprint = fq.fq_set_config([int(b) for b in bits])
+
+    # activations: one seeded fp16 vector per matrix; host copies are pinned for the end-to-end leg
+    k_off = np.concatenate([[0], np.cumsum([s.k_in for s in shapes])])
+    n_off = np.concatenate([[0], np.cumsum([s.n_out for s in shapes])])
+    x_host = torch.empty(int(k_off[-1]), dtype=torch.float16).pin_memory()
+    for i, sh in enumerate(shapes):
+        x_host[k_off[i]:k_off[i + 1]] = S.activations(S.tensor_key(CONFIG_ID, i, S.TENSOR_X), 1, sh.k_in)[0]
+    y_host = torch.empty(int(n_off[-1]), dtype=torch.float16).pin_memory()
+    x_dev = x_host.to(device)
+    y_dev = torch.zeros(int(n_off[-1]), dtype=torch.float16, device=device)
+    xs = [x_dev[k_off[i]:k_off[i + 1]] for i in range(L)]
+    ys = [y_dev[n_off[i]:n_off[i + 1]] for i in range(L)]
+    layers = list(range(L))
+    args_dep = fq.stack_args(layers, xs, ys, phases)
+    args_free = fq.stack_args(layers, xs, ys, None)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def step_dev():
+        fq.fq_gemv_stack_raw(args_dep, 1)
+
+    def step_free():
+        fq.fq_gemv_stack_raw(args_free, 1)
+
+    def step_e2e():
+        x_dev.copy_(x_host, non_blocking=True)
+        fq.fq_gemv_stack_raw(args_dep, 1)
+        y_host.copy_(y_dev, non_blocking=True)
+
+    for _ in range(args.warmup):
+        step_dev()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms = timed(step_dev, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    for _ in range(3):
+        step_free()
+    ms_free = timed(step_free, args.steps)
+    for _ in range(3):
+        step_e2e()
+    ms_e2e = timed(step_e2e, args.steps)
+    status = fq.fq_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the timed region")
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = measured_peaks()
+    gbs = footprint / (ms * 1e-3) / 1e9
+    traffic, traffic_note = read_ncu_traffic(footprint)
+    line = {
+        "metric": METRIC, "value": gbs * world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {
+            "workload": f"llama2-7b-shaped decode stack: {L} matrices ({args.blocks} blocks), per-matrix bits seeded from "
+                        f"{BIT_CHOICES}, g=128, packed format, batch-1 fp16 GEMV, one persistent launch per pass, "
+                        f"dependency phases honoured",
+            "average_bits": S.average_bits(bits, shapes), "footprint_bytes": footprint,
+            "l2": "each pass streams the whole stack (>> 126 MB L2), no flush needed",
+            "replicas": world,
+        },
+        "e2e": {"value": footprint / (ms_e2e * 1e-3) / 1e9 * world, "unit": UNIT,
+                "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(y_host.numel() * 2),
+                "ms_per_step": ms_e2e},
+        "gpu_launches": args.steps,
+        "unordered": {"value": footprint / (ms_free * 1e-3) / 1e9 * world, "unit": UNIT, "ms_per_step": ms_free,
+                      "note": "same pass without the dependency phases (every matrix independent)"},
+        "roofline": {
+            "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": gbs / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
+            "frac_of_nominal_8TBs": gbs / 8000.0,
+            "kernel": "gemv_kernel<1> (one launch per pass; algorithmic bytes = footprint of the configuration)",
+            "traffic": traffic, "traffic_note": traffic_note,
+        },
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline:
+        n_layers = min(args.ref_layers, L)
+        byts, secs, desc = oracle_sample(shapes, bits, n_layers, device)
+        line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+    print(json.dumps(line), flush=True)
+    fq.fq_destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
