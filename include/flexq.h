@@ -46,7 +46,8 @@ enum { FQ_OK = 0,
        FQ_ERR_NO_VARIANT = -5,  /* configuration asks for a bit-width that is not stored    */
        FQ_ERR_NOT_PACKED = -6,  /* layer used before fq_pack_layer / fq_set_config          */
        FQ_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, out of memory...) */
-       FQ_ERR_TIMEOUT = -8 };   /* a bounded device-side wait ran out (see fq_status)       */
+       FQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait ran out (see fq_status)       */
+       FQ_ERR_SCRATCH = -9 };   /* problem needs more than the built-in scratch (fq_gemv_static) */
 
 #define FQ_MAX_BATCH 8          /* decode batch handled by the GEMV family */
 
@@ -105,6 +106,27 @@ int fq_set_config(fq_ctx* ctx, const uint8_t* bits_host, int n_layers,
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.
  * Enqueues kernels on `stream`; does not synchronise. */
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
+
+/* Same result as fq_gemv, for callers that must not allocate device memory.  (The paper has no
+ * counterpart; this is a deployment convenience.)  fq_gemv may grow the context's workspace
+ * with cudaMalloc when a layer needs more split-K scratch than any earlier call did.  That is
+ * not acceptable for callers such as a real-time serving loop with a fixed memory budget, code
+ * running while another library owns the allocator, or a host thread that must never block on
+ * the device-wide synchronisation an allocation implies.  This variant keeps its split-K
+ * scratch (per-row-tile arrival counters and fp32 partial sums) in a fixed array that is part
+ * of the library image: FQ_STATIC_SCRATCH_BYTES on every GPU that loads the library, held
+ * until the process exits.  It calls no cudaMalloc / cudaFree and nothing that allocates.
+ *   - batch 1 only; x_dev fp16 [k_in], y_dev fp16 [n_out], 16-byte aligned, caller-owned.
+ *   - Returns FQ_ERR_SCRATCH (and launches nothing) when the layer at its active width needs
+ *     more scratch than the array holds: 4 bytes per 16-row tile plus 64 bytes per
+ *     (16-row tile x K chunk).  Every Llama-2-7B / 13B shaped layer fits.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left there; the
+ *     counters are cleared on `stream` before each launch.  Two calls that overlap on the GPU
+ *     (different streams, or different contexts) race on it: serialise them. */
+#define FQ_STATIC_SCRATCH_BYTES (1u << 20)
+int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
 
 /* Decode at batch 1..8:  Y[b][n] = sum_k X[b][k] * w^[n][k].
  *   x_dev fp16 [batch][k_in], y_dev fp16 [batch][n_out], densely packed rows. */

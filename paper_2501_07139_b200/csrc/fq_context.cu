@@ -123,6 +123,7 @@ const char* fq_strerror(int code)
         case FQ_ERR_NOT_PACKED: return "layer not packed";
         case FQ_ERR_CUDA: return "CUDA runtime error";
         case FQ_ERR_TIMEOUT: return "device-side wait timed out";
+        case FQ_ERR_SCRATCH: return "layer needs more than the built-in scratch";
         default: return "unknown error";
     }
 }
@@ -302,6 +303,17 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream)
 {
     return fq_gemv_batched(ctx, layer, x_dev, 1, y_dev, stream);
+}
+
+int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream)
+{
+    if (!ctx) return FQ_ERR_ARG;
+    GemvOp op;
+    const int rc = fill_op(ctx, layer, x_dev, y_dev, 1, op);
+    if (rc != FQ_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    return launch_gemv_static(ctx, op, op_counter_bytes(op), op_partial_bytes(op, 1), (cudaStream_t)stream);
 }
 
 int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t* const* x_dev_host,

@@ -514,4 +514,44 @@ int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, i
     return max_batch <= 1 ? launch_impl<1>(ctx, dummy, sa, coop, st) : launch_impl<8>(ctx, dummy, sa, coop, st);
 }
 
+// ------------------------------------------------------------------------------- allocation-free variant
+// Split-K scratch that is part of the library image, for callers that must not allocate.
+// Host code may only use the symbol through cudaGetSymbolAddress (its name is not a device
+// address on the host side).
+static __device__ __align__(256) unsigned char g_static_scratch[FQ_STATIC_SCRATCH_BYTES];
+
+static int static_scratch_address(int device, unsigned char** out)
+{
+    static unsigned char* addr[64] = {};
+    if (device < 0 || device >= 64) return FQ_ERR_ARG;
+    if (!addr[device]) {                       // once per device, with that device current
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return FQ_ERR_CUDA;
+        addr[device] = static_cast<unsigned char*>(p);
+    }
+    *out = addr[device];
+    return FQ_OK;
+}
+
+// Runs one batch-1 decode op with counters and partials placed in the built-in array.
+int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st)
+{
+    const size_t counters = (size_t)round_up((int64_t)counter_bytes, 256);
+    if (counters + partial_bytes > FQ_STATIC_SCRATCH_BYTES) return FQ_ERR_SCRATCH;
+    unsigned char* base = nullptr;
+    const int rc = static_scratch_address(ctx->device, &base);
+    if (rc != FQ_OK) return rc;
+    op.tile_count = reinterpret_cast<unsigned*>(base);
+    op.partial = reinterpret_cast<float*>(base + counters);
+    // the array keeps the previous call's contents: arrival counters must start at zero
+    if (counter_bytes) FQ_CUDA_OK(cudaMemsetAsync(base, 0, counter_bytes, st));
+    StackArgs sa{};
+    sa.table = nullptr;
+    sa.status = ctx->status_dev;
+    sa.n_ops = 1;
+    sa.n_phases = 0;
+    sa.total_units = (long long)op.n_rt * op.n_chunks;
+    return launch_impl<1>(ctx, op, sa, false, st);
+}
+
 }  // namespace fq

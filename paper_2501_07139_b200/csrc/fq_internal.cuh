@@ -86,6 +86,7 @@ int launch_export_meta(const void* meta, int n_out, int k_in, uint16_t* scales, 
 int gemv_chunks(int n_ss, int bits, int batch);
 size_t gemv_partial_floats_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
+int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st);
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
 
 }  // namespace fq

@@ -22,7 +22,7 @@ _lib = None
 EXPORTS = [
     "fq_create", "fq_destroy", "fq_code_bytes", "fq_meta_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
-    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror",
+    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static",
 ]
 
 
@@ -57,6 +57,7 @@ def lib():
     L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
     L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
+    L.fq_gemv_static.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_stack.argtypes = [vp, i, vp, vp, vp, vp, i, vp]
     L.fq_gemm.argtypes = [vp, i, vp, i, i, vp, i, vp]
     L.fq_export_layer.argtypes = [vp, i, i, vp, vp]
@@ -176,6 +177,12 @@ class FlexQ:
     # -- decode --------------------------------------------------------------------------
     def fq_gemv(self, layer: int, x: torch.Tensor, y: torch.Tensor):
         _check(lib().fq_gemv(self._h, layer, x.data_ptr(), y.data_ptr(), _stream()), "fq_gemv")
+        return y
+
+    def fq_gemv_static(self, layer: int, x: torch.Tensor, y: torch.Tensor):
+        """fq_gemv without any device allocation: split-K scratch lives in a fixed array inside the
+        library (see include/flexq.h).  Raises FlexQError(-9) when the layer does not fit."""
+        _check(lib().fq_gemv_static(self._h, layer, x.data_ptr(), y.data_ptr(), _stream()), "fq_gemv_static")
         return y
 
     def fq_gemv_batched(self, layer: int, x: torch.Tensor, y: torch.Tensor):
