@@ -65,21 +65,25 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.k_in = L.k_in;
     op.n_rt = row_tiles(L.n_out);
     op.n_ss = supersteps(L.k_in);
-    op.n_chunks = gemv_chunks(op.n_ss, bits, batch);
+    op.n_rp = (op.n_rt + kUnitRowTiles - 1) / kUnitRowTiles;
+    op.chunk_steps = gemv_chunk_steps(bits, batch);
+    op.n_chunks = (op.n_ss + op.chunk_steps - 1) / op.chunk_steps;
     op.batch = batch;
     // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
-    op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (float)(1 << (7 - bits)) : 0.f;
+    op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
+    op.n_units = op.n_chunks * op.n_rp;
+    if ((long long)op.n_chunks * op.n_rp * 1024 >= (1ll << 31)) return FQ_ERR_SHAPE;   // 32-bit unit arithmetic on the device
     op.phase = -1;
-    op.unit_base = 0;
+    op.rot = 0;
     return FQ_OK;
 }
 
 size_t op_partial_bytes(const GemvOp& op, int max_batch)
 {
     if (op.n_chunks <= 1) return 0;
-    return (size_t)op.n_rt * op.n_chunks * gemv_partial_floats_per_unit(max_batch) * sizeof(float);
+    return (size_t)op.n_rp * op.n_chunks * gemv_partial_floats_per_unit(max_batch) * sizeof(float);
 }
-size_t op_counter_bytes(const GemvOp& op) { return op.n_chunks <= 1 ? 0 : (size_t)round_up(op.n_rt * 4, 16); }
+size_t op_counter_bytes(const GemvOp& op) { return op.n_chunks <= 1 ? 0 : (size_t)round_up(op.n_rp * 4, 16); }
 
 uint64_t hash_mix(uint64_t h, uint64_t v)
 {
@@ -343,7 +347,8 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         key = hash_mix(key, (uint64_t)reinterpret_cast<uintptr_t>(y_dev_host[i]));
         key = hash_mix(key, phases_host ? (uint64_t)phases_host[i] : ~0ull);
     }
-    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) + (size_t)(n_phases > 0 ? n_phases : 1) * sizeof(long long);
+    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) + (size_t)(n_phases > 0 ? n_phases : 1) * sizeof(long long) +
+                               (size_t)ctx->sm_count * sizeof(int);
     const size_t hdr_off = (size_t)round_up((int64_t)table_bytes, 16);
     StackHeader hdr{};
 
@@ -360,12 +365,13 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         for (int p = 0; p < (n_phases > 0 ? n_phases : 1); p++) phase_total[p] = 0;
         size_t ws_need = kWsHead;
         long long unit_base = 0;
+        std::vector<long long> bases(n_ops);
         for (int i = 0; i < n_ops; i++) {
             const int rc = fill_op(ctx, layers_host[i], x_dev_host[i], y_dev_host[i], batch, ops[i]);
             if (rc != FQ_OK) return rc;
             ops[i].phase = phases_host ? phases_host[i] : -1;
-            ops[i].unit_base = unit_base;
-            const long long units = (long long)ops[i].n_rt * ops[i].n_chunks;
+            bases[i] = unit_base;
+            const long long units = (long long)ops[i].n_rp * ops[i].n_chunks;
             unit_base += units;
             if (phases_host) phase_total[phases_host[i]] += units;
             ws_need = (size_t)round_up((int64_t)ws_need, 256);
@@ -384,6 +390,17 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             ops[i].partial = reinterpret_cast<float*>(ctx->ws + off);
             off += op_partial_bytes(ops[i], batch);
         }
+        // how many units each CTA of the persistent grid will see (the consumers' loop bound)
+        int* cta_units = reinterpret_cast<int*>(phase_total + (n_phases > 0 ? n_phases : 1));
+        const int grid = (int)(unit_base < ctx->sm_count ? unit_base : ctx->sm_count);
+        for (int i = 0; i < n_ops; i++) ops[i].rot = (int)(bases[i] % (grid > 0 ? grid : 1));
+        for (int c = 0; c < ctx->sm_count; c++) cta_units[c] = 0;
+        for (int i = 0; i < n_ops; i++)
+            for (int c = 0; c < grid; c++) {
+                int lo, hi;
+                gemv_cta_range(ops[i].n_units, ops[i].rot, c, grid, lo, hi);
+                cta_units[c] += hi - lo;
+            }
         hdr.n_ops = n_ops; hdr.n_phases = n_phases; hdr.total_units = unit_base;
         std::memcpy(ctx->stack_host + hdr_off, &hdr, sizeof hdr);
         if (ctx->stack_dev_bytes < table_bytes) {

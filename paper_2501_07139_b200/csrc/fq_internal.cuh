@@ -23,6 +23,8 @@ struct Layer {
     Variant var[9];              // PACKED: index = bits; PLANES: only [8]
 };
 
+constexpr int kUnitRowTiles = 2;   // a decode unit covers two 16-row tiles (32 output rows)
+
 // What one decode op needs on the device.
 struct GemvOp {
     const uint8_t* field_ptr[kMaxFields];
@@ -34,14 +36,17 @@ struct GemvOp {
     const uint16_t* x;           // fp16 [batch][k_in]
     uint16_t* y;                 // fp16 [batch][n_out]
     float* partial;              // split-K partial sums (unused when n_chunks == 1)
-    unsigned* tile_count;        // split-K arrival counters, one per row tile
+    unsigned* tile_count;        // split-K arrival counters, one per row pair
     int n_out, k_in;
     int n_rt, n_ss;              // row tiles, supersteps
-    int n_chunks;                // K chunks per row tile
+    int n_rp;                    // row pairs = units per K chunk
+    int n_chunks;                // K chunks
+    int chunk_steps;             // supersteps per K chunk (the last chunk may be shorter)
     int batch;
-    float zero_adjust;           // subtracted from every zero point (mid-point fill of a nested child)
+    int zero_adjust;             // subtracted from every zero point (mid-point fill of a nested child)
     int phase;                   // -1: no ordering
-    long long unit_base;         // global index of this op's first unit
+    int n_units;                 // n_chunks * n_rp
+    int rot;                     // rotation of the CTA blocks for this op (evens out remainders)
 };
 
 struct StackHeader {
@@ -82,12 +87,15 @@ int launch_export_planes(const void* codes, int n_out, int k_in, int bits, const
                          uint32_t* out, cudaStream_t st);
 int launch_export_meta(const void* meta, int n_out, int k_in, uint16_t* scales, uint16_t* zeros, cudaStream_t st);
 
-// Chunking policy of the decode kernel: number of K chunks per row tile.
-int gemv_chunks(int n_ss, int bits, int batch);
+// Chunking policy of the decode kernel: supersteps (256 columns) per K chunk.
+int gemv_chunk_steps(int bits, int batch);
 size_t gemv_partial_floats_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
 int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st);
+// table_dev: [GemvOp x n_ops][long long phase_total x max(n_phases,1)][int cta_units x sm_count]
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
+// Units of an op (n_units units, block rotation rot) that CTA `cta` of `grid` processes: [lo, hi).
+void gemv_cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi);
 
 }  // namespace fq
 

@@ -8,10 +8,12 @@
 // Every array is tiled: tile = 16 rows x 256 columns ("superstep"), tiles ordered
 // [row_tile][superstep], and inside a tile  [f chunks][32 lanes][16 bytes].
 // The order inside a tile is the order in which a warp consumes the values as A-operand
-// registers of mma.m16n8k16 (lane = 4*g + c owns rows g, g+8 and columns 32*j2 + 8*c + i):
-// each 32-bit word holds 16/f "pair registers"; pair register t is the two fields at bit
-// offsets t*f (low half) and 16 + t*f (high half), so one shift and one AND turn a stored
-// word into a ready half2 operand whose halves hold the integers as fp16 subnormals.
+// registers of the 8-bit mma.m16n8k32 (lane = 4*g + c owns rows g, g+8; in k32 step j it owns
+// columns 32j + 4c .. +3 and 32j + 16 + 4c .. +3).  A 32-bit word holds P = 8/f A-registers
+// on top of each other: byte b of the word belongs to k-slot b, and inside every byte the
+// field of register t sits at bit offset t*f.  So `word & (field_mask << t*f)` IS the A
+// register of k32 step  j = P*chunk + t  (values scaled by 2^(t*f)), with no shift at all;
+// the four words of a lane's 16-byte chunk are the four A registers a0..a3.
 //
 // Metadata: [row_tile][group][16 rows] words, low half = scale, high half = zero (fp16).
 #pragma once
@@ -81,31 +83,30 @@ struct FieldPos { int word_byte; int bit; };
 
 FQ_HD FieldPos field_pos(int f, int r, int kk)
 {
+    const int P = 8 / f;                                      // A-registers stacked in one word
     const int g = r & 7, hi_row = r >> 3;
-    const int j2 = kk >> 5, c = (kk >> 3) & 3, i = kk & 7;
-    const int mma = i >> 2, pair = (i >> 1) & 1, half = i & 1;
-    const int reg = j2 * 8 + mma * 4 + pair * 2 + hi_row;     // 0..63: A-register of this lane in the superstep
-    const int regs_per_chunk = 64 / f;
-    const int regs_per_word = 16 / f;
-    const int chunk = reg / regs_per_chunk;
-    const int rr = reg % regs_per_chunk;
-    const int word = rr / regs_per_word;
-    const int t = rr % regs_per_word;
-    FieldPos p;
-    p.word_byte = chunk * 512 + (4 * g + c) * 16 + word * 4;
-    p.bit = half * 16 + t * f;
-    return p;
+    const int j = kk >> 5, p = kk & 31;
+    const int half = p >> 4, c = (p >> 2) & 3, byte = p & 3;
+    const int chunk = j / P, t = j % P;
+    const int areg = 2 * half + hi_row;                       // a0..a3 of the mma
+    FieldPos q;
+    q.word_byte = chunk * 512 + (4 * g + c) * 16 + areg * 4;
+    q.bit = byte * 8 + t * f;
+    return q;
 }
 
-// Inverse: which (row, column) of the tile does bit field (half, t) of word `word` of lane
-// `lane` of chunk `chunk` belong to.
-FQ_HD void field_owner(int f, int chunk, int lane, int word, int half, int t, int& r, int& kk)
+// Inverse: field slot q (0 .. 32/f - 1; q = byte * P + t) of word `word` of lane `lane` of chunk
+// `chunk` belongs to which (row, column) of the tile, and at which bit it sits.
+FQ_HD void field_owner(int f, int chunk, int lane, int word, int q, int& r, int& kk, int& bit)
 {
-    const int reg = chunk * (64 / f) + word * (16 / f) + t;
-    const int j2 = reg >> 3, mma = (reg >> 2) & 1, pair = (reg >> 1) & 1, hi_row = reg & 1;
+    const int P = 8 / f;
+    const int byte = q / P, t = q % P;
     const int g = lane >> 2, c = lane & 3;
+    const int half = word >> 1, hi_row = word & 1;
+    const int j = chunk * P + t;
     r = g + 8 * hi_row;
-    kk = j2 * 32 + c * 8 + mma * 4 + pair * 2 + half;
+    kk = j * 32 + half * 16 + c * 4 + byte;
+    bit = byte * 8 + t * f;
 }
 
 }  // namespace fq

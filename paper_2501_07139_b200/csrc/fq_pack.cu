@@ -117,16 +117,15 @@ __global__ void __launch_bounds__(256) pack_kernel(const PackArgs a)
         const int rt = (int)(tile / a.n_ss), ss = (int)(tile % a.n_ss);
         const unsigned mask = (1u << f) - 1u;
         unsigned v = 0;
-        for (int half = 0; half < 2; half++)
-            for (int t = 0; t < 16 / f; t++) {
-                int r, kk;
-                field_owner(f, chunk, lane, word, half, t, r, kk);
-                const long long n = (long long)rt * kTileRows + r;
-                const long long k = (long long)ss * kStepCols + kk;
-                unsigned code = 0;
-                if (n < a.n_out && k < a.k_in) code = a.codes[n * a.k_in + k];
-                v |= ((code >> sh) & mask) << (half * 16 + t * f);
-            }
+        for (int q = 0; q < 32 / f; q++) {
+            int r, kk, bit;
+            field_owner(f, chunk, lane, word, q, r, kk, bit);
+            const long long n = (long long)rt * kTileRows + r;
+            const long long k = (long long)ss * kStepCols + kk;
+            unsigned code = 0;
+            if (n < a.n_out && k < a.k_in) code = a.codes[n * a.k_in + k];
+            v |= ((code >> sh) & mask) << bit;
+        }
         a.out[wi] = v;
     }
 }
