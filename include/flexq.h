@@ -56,13 +56,12 @@ int fq_create(fq_ctx** out, int device, int n_layers);
 /* Frees the context and its workspace.  Caller-owned buffers are not touched. */
 int fq_destroy(fq_ctx* ctx);
 
-/* Bytes the caller must allocate for the code buffer of one stored variant.  The device
- * layout is tiled (16 rows x 256 columns), so this is the algorithmic size
- * n_out*k_in*bits/8 (PACKED) or n_out*k_in (PLANES: the 8-bit parent) computed on
- * n_out rounded up to 16 and k_in rounded up to 256.  Returns 0 on invalid arguments. */
-size_t fq_code_bytes(int n_out, int k_in, int bits, int fmt);
-/* Bytes for the scale/zero buffer of a layer (4 bytes per group, same rounding). */
-size_t fq_meta_bytes(int n_out, int k_in, int group);
+/* Bytes the caller must allocate for one stored variant: codes AND scale/zero words, which the
+ * device layout interleaves (blobs of 32 rows x 512 columns) so that a decode step fetches both
+ * with one copy.  This is the algorithmic size n_out*k_in*bits/8 + n_out*(k_in/128)*4
+ * (bits = 8 for a PLANES parent) computed on n_out rounded up to 32 and k_in rounded up to 512.
+ * Returns 0 on invalid arguments. */
+size_t fq_store_bytes(int n_out, int k_in, int bits, int fmt);
 
 /* Min-max asymmetric group quantiser (the step in front of the path; the paper takes the
  * quantised models QM(n) of Sec. III-A as given).  Per group of 128 columns, in double:
@@ -80,16 +79,15 @@ int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int gro
  *   PACKED: `bits` in [2,8] is the width of this variant; call again with another width
  *           to add a variant of the same layer (same shape).
  *   PLANES: `bits` must be 8; the parent is stored as a 2-bit top field plus six 1-bit
- *           planes, most significant first, so a b-bit child reads exactly the first b/8
- *           of the buffer and every b in [2,8] becomes selectable.
+ *           planes, most significant first inside every blob, so a b-bit child reads exactly
+ *           the first b/8 of every blob's codes and every b in [2,8] becomes selectable.
  *   codes_dev   uint8 [n_out][k_in], one code per byte; read, not retained.
  *   scales_dev, zeros_dev   fp16 [n_out][k_in/128]; read, not retained.
- *   code_out_dev  fq_code_bytes() bytes, 256-byte aligned; written and RETAINED.
- *   meta_out_dev  fq_meta_bytes() bytes, 256-byte aligned; written and RETAINED.
+ *   store_out_dev fq_store_bytes() bytes, 256-byte aligned; written and RETAINED.
  * The first variant packed for a layer becomes its active one. */
 int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int group, int fmt,
                   const uint8_t* codes_dev, const uint16_t* scales_dev, const uint16_t* zeros_dev,
-                  void* code_out_dev, void* meta_out_dev, void* stream);
+                  void* store_out_dev, void* stream);
 
 /* Activates an elastic configuration (Sec. III-A: an EQM is a per-module choice among the
  * stored variants; Sec. II-C: switching should cost as little memory traffic as possible).

@@ -49,25 +49,24 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     if (!v) return FQ_ERR_NO_VARIANT;
     const FieldList fl = active_fields(L, bits);
     std::memset(&op, 0, sizeof op);
-    const uint8_t* p = static_cast<const uint8_t*>(v->codes);
     for (int i = 0; i < fl.n; i++) {
-        op.field_ptr[i] = p;
         op.field_width[i] = fl.width[i];
         op.field_shift[i] = fl.shift[i];
-        p += field_bytes(L.n_out, L.k_in, fl.width[i]);
     }
     op.n_fields = fl.n;
     op.bits = bits;
-    op.meta = static_cast<const uint32_t*>(v->meta);
+    op.store = static_cast<const uint8_t*>(v->store);
+    op.blob_stride = blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits);
+    op.blob_read = blob_bytes(bits);
     op.x = x;
     op.y = y;
     op.n_out = L.n_out;
     op.k_in = L.k_in;
-    op.n_rt = row_tiles(L.n_out);
     op.n_ss = supersteps(L.k_in);
-    op.n_rp = (op.n_rt + kUnitRowTiles - 1) / kUnitRowTiles;
-    op.chunk_steps = gemv_chunk_steps(bits, batch);
-    op.n_chunks = (op.n_ss + op.chunk_steps - 1) / op.chunk_steps;
+    op.n_kb = k_blobs(L.k_in);
+    op.n_rp = row_pairs(L.n_out);
+    op.chunk_blobs = gemv_chunk_blobs(bits, batch);
+    op.n_chunks = (op.n_kb + op.chunk_blobs - 1) / op.chunk_blobs;
     op.batch = batch;
     // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
     op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
@@ -172,19 +171,13 @@ int fq_destroy(fq_ctx* ctx)
     return FQ_OK;
 }
 
-size_t fq_code_bytes(int n_out, int k_in, int bits, int fmt)
+size_t fq_store_bytes(int n_out, int k_in, int bits, int fmt)
 {
     if (n_out < 1 || k_in < 1 || k_in % kGroup != 0) return 0;
     if (fmt == FQ_FMT_PLANES) { if (bits != 8) return 0; }
     else if (fmt == FQ_FMT_PACKED) { if (bits < 2 || bits > 8) return 0; }
     else return 0;
-    return (size_t)row_tiles(n_out) * supersteps(k_in) * 512 * bits;
-}
-
-size_t fq_meta_bytes(int n_out, int k_in, int group)
-{
-    if (n_out < 1 || k_in < 1 || group != kGroup || k_in % kGroup != 0) return 0;
-    return (size_t)row_tiles(n_out) * supersteps(k_in) * 2 * 16 * 4;
+    return (size_t)store_bytes(n_out, k_in, bits);
 }
 
 int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int group,
@@ -199,26 +192,26 @@ int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int gro
 
 int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int group, int fmt,
                   const uint8_t* codes_dev, const uint16_t* scales_dev, const uint16_t* zeros_dev,
-                  void* code_out_dev, void* meta_out_dev, void* stream)
+                  void* store_out_dev, void* stream)
 {
-    if (!ctx || !codes_dev || !scales_dev || !zeros_dev || !code_out_dev || !meta_out_dev) return FQ_ERR_ARG;
+    if (!ctx || !codes_dev || !scales_dev || !zeros_dev || !store_out_dev) return FQ_ERR_ARG;
     if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
     if (fmt != FQ_FMT_PACKED && fmt != FQ_FMT_PLANES) return FQ_ERR_ARG;
     if (bits < 2 || bits > 8 || (fmt == FQ_FMT_PLANES && bits != 8)) return FQ_ERR_BITS;
     if (group != kGroup || n_out < 1 || k_in < 1 || k_in % kGroup != 0) return FQ_ERR_SHAPE;
-    if (!aligned(code_out_dev, 256) || !aligned(meta_out_dev, 256)) return FQ_ERR_ALIGN;
+    if (!aligned(store_out_dev, 256)) return FQ_ERR_ALIGN;
     Layer& L = ctx->layers[layer];
     if (L.registered && (L.n_out != n_out || L.k_in != k_in || L.fmt != fmt)) return FQ_ERR_SHAPE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
     const FieldList fl = fmt == FQ_FMT_PLANES ? plane_fields(8) : packed_fields(bits);
-    const int rc = launch_pack(codes_dev, scales_dev, zeros_dev, n_out, k_in, fl, code_out_dev, meta_out_dev,
+    const int rc = launch_pack(codes_dev, scales_dev, zeros_dev, n_out, k_in, bits, fl, store_out_dev,
                                (cudaStream_t)stream);
     if (rc != FQ_OK) return rc;
     L.registered = true;
     L.n_out = n_out; L.k_in = k_in; L.fmt = fmt;
     Variant& v = L.var[bits];
-    v.present = true; v.codes = code_out_dev; v.meta = meta_out_dev;
+    v.present = true; v.store = store_out_dev;
     if (L.active_bits == 0) L.active_bits = bits;
     ctx->config_epoch++;
     return FQ_OK;
@@ -438,9 +431,9 @@ int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* strea
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
     if (L.fmt == FQ_FMT_PLANES)
-        return launch_export_planes(v->codes, L.n_out, L.k_in, bits, plane_fields(bits), (uint32_t*)out_dev,
+        return launch_export_planes(v->store, L.n_out, L.k_in, bits, plane_fields(bits), (uint32_t*)out_dev,
                                     (cudaStream_t)stream);
-    return launch_export_packed(v->codes, L.n_out, L.k_in, bits, packed_fields(bits), (uint32_t*)out_dev,
+    return launch_export_packed(v->store, L.n_out, L.k_in, bits, packed_fields(bits), (uint32_t*)out_dev,
                                 (cudaStream_t)stream);
 }
 
@@ -454,7 +447,8 @@ int fq_export_meta(fq_ctx* ctx, int layer, int bits, uint16_t* scales_dev, uint1
     if (!v) return FQ_ERR_NO_VARIANT;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
-    return launch_export_meta(v->meta, L.n_out, L.k_in, scales_dev, zeros_dev, (cudaStream_t)stream);
+    return launch_export_meta(v->store, L.n_out, L.k_in, L.fmt == FQ_FMT_PLANES ? 8 : bits, scales_dev, zeros_dev,
+                              (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -35,32 +35,32 @@ namespace fq {
 #define FQ_GEMV_WARPS 8
 #endif
 #ifndef FQ_GEMV_UNIT_BYTES
-#define FQ_GEMV_UNIT_BYTES 16384
+#define FQ_GEMV_UNIT_BYTES 17408
 #endif
 constexpr int kConsumerWarps = FQ_GEMV_WARPS;
 constexpr int kProducerWarp = kConsumerWarps;          // warp index of the producer
 constexpr int kPrepWarp = kConsumerWarps + 1;          // first warp of the activation pre-processors
 constexpr int kPrepWarps = 4;                          // they share the items of a segment
 constexpr int kGemvThreads = (kConsumerWarps + 1 + kPrepWarps) * 32;
-constexpr int kUnitCodeBytes = FQ_GEMV_UNIT_BYTES;     // code bytes of one unit, at most
+constexpr int kUnitBytes = FQ_GEMV_UNIT_BYTES;         // bytes of one unit (whole blobs), at most: 2 x 4-bit or 1 x 8-bit blob
 constexpr int kXSlots = 4;                             // activation chunks kept in shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 template <int MAXB> struct GemvCfg;
-template <> struct GemvCfg<1> { static constexpr int kCMax = 8; };      // supersteps per chunk, at most
-template <> struct GemvCfg<8> { static constexpr int kCMax = 2; };
+template <> struct GemvCfg<1> { static constexpr int kBlobsMax = 3; };  // k blobs (512 columns) per chunk, at most
+template <> struct GemvCfg<8> { static constexpr int kBlobsMax = 1; };
 
 // What the producer tells the consumers: once per op a copy of the op descriptor in a ring ...
 constexpr int kOpRing = 32;                            // > stages: an op slot outlives its last unit
 // ... and once per unit (next to the stage that holds the unit's weights)
 struct UnitDesc {
-    int ch, rp, cnt, n_tiles, seg, op_slot, pad[2];
+    int ch, rp, nb, seg, op_slot, pad[3];       // K chunk, row pair, blobs in the unit, activation segment, op ring slot
 };
 static_assert(sizeof(UnitDesc) == 32, "descriptor layout");
 
 template <int MAXB> struct GemvSmem {
-    static constexpr int kCMax = GemvCfg<MAXB>::kCMax;
-    static constexpr int kStageBytes = kUnitCodeBytes + kUnitRowTiles * kCMax * 128;
+    static constexpr int kCMax = GemvCfg<MAXB>::kBlobsMax * kBlobSteps;     // supersteps per chunk, at most
+    static constexpr int kStageBytes = kUnitBytes;
     // activation slot: low digits, high digits (rows padded so that LDS.64 of a quarter warp is
     // conflict free), then per (row, group) the integer sum and the power-of-two scale
     static constexpr int kXRow = MAXB == 1 ? kCMax * 256 : kCMax * 256 + 32;
@@ -88,15 +88,16 @@ template <int MAXB> struct GemvSmem {
     static_assert(kTotal <= 232448, "decode kernel: shared memory over the 227 KB per-CTA limit");
 };
 
-// Supersteps (256 columns) per K chunk for a variant of `bits` bits.
-int gemv_chunk_steps(int bits, int batch)
+// K blobs (512 columns) per K chunk for a variant of which `bits` bits are read.
+int gemv_chunk_blobs(int bits, int batch)
 {
-    const int cmax = batch <= 1 ? GemvCfg<1>::kCMax : GemvCfg<8>::kCMax;
-    int c = kUnitCodeBytes / (kUnitRowTiles * 512 * bits);
+    const int cmax = batch <= 1 ? GemvCfg<1>::kBlobsMax : GemvCfg<8>::kBlobsMax;
+    int c = kUnitBytes / blob_bytes(bits);
     if (c > cmax) c = cmax;
     if (c < 1) c = 1;
     return c;
 }
+static_assert(kUnitBytes >= kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * 8, "a unit must hold an 8-bit blob");
 
 size_t gemv_partial_floats_per_unit(int batch) { return batch <= 1 ? 32 : 256; }
 
@@ -352,29 +353,20 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 op_seq++;
                 const int op_slot = op_seq % kOpRing;
                 cur.store(reinterpret_cast<GemvOp*>(opring + op_slot * S::kOpBytes), lane);   // for the consumers
-                // this lane's copy: lanes 2*fi + t -> field fi of tile t; lanes 2*n_fields + t -> scale/zero of tile t
-                const int my_t = lane & 1, my_f = lane >> 1;
-                const bool is_field = my_f < op.n_fields, is_meta = my_f == op.n_fields;
-                int fw = 0, prefix = 0;                               // my field's width, widths before it
-                if (is_field) {
-                    fw = op.field_width[my_f];
-                    for (int i = 0; i < my_f; i++) prefix += op.field_width[i];
-                }
-                const uint8_t* src_base = is_field ? op.field_ptr[my_f] : reinterpret_cast<const uint8_t*>(op.meta);
-                const int bytes_per_step = is_field ? fw * 512 : 128; // my source bytes per (tile, superstep)
+                // a PACKED variant's blobs are contiguous: one copy per unit (lane 0); a nested child reads a
+                // prefix of every blob: one copy per blob (lanes 0 .. nb-1)
+                const bool contiguous = op.blob_read == op.blob_stride;
                 const int n_units = hi - lo;
                 int ch = lo / op.n_rp, rp = lo % op.n_rp;
                 bool new_chunk = true;
-                int ss0 = 0, cnt = 0;
+                int kb0 = 0, nb = 0;
                 for (int iu = 0; iu < n_units; iu++) {
                     if (new_chunk) {
                         seg++;
-                        ss0 = ch * op.chunk_steps;
-                        cnt = min(op.chunk_steps, op.n_ss - ss0);
+                        kb0 = ch * op.chunk_blobs;
+                        nb = min(op.chunk_blobs, op.n_kb - kb0);
                         new_chunk = false;
                     }
-                    const int rt0 = rp * kUnitRowTiles;
-                    const int n_tiles = min(kUnitRowTiles, op.n_rt - rt0);
                     const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
                     int ok = 1;
                     if (lane == 0) {
@@ -386,19 +378,18 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                         }
                         if (ok) {
                             UnitDesc* d = reinterpret_cast<UnitDesc*>(smem + S::oDesc) + stage;
-                            d->ch = ch; d->rp = rp; d->cnt = cnt; d->n_tiles = n_tiles; d->seg = seg; d->op_slot = op_slot;
-                            mbar_expect_tx(full, (uint32_t)(n_tiles * cnt) * (512u * op.bits + 128u));
+                            d->ch = ch; d->rp = rp; d->nb = nb; d->seg = seg; d->op_slot = op_slot;
+                            mbar_expect_tx(full, (uint32_t)(nb * op.blob_read));
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) { stop = true; break; }
-                    // stage layout: [field][tile][cnt * f * 512 B] ... then [tile][cnt * 128 B] of scale/zero
-                    if (my_t < n_tiles && (is_field || is_meta)) {
-                        const uint32_t stage_base = smem_u32(smem + S::oStages + stage * S::kStageBytes);
-                        const uint32_t dst = is_field ? stage_base + cnt * 512 * (n_tiles * prefix + my_t * fw)
-                                                      : stage_base + cnt * 512 * n_tiles * op.bits + my_t * cnt * 128;
-                        const long long tile0 = (long long)(rt0 + my_t) * op.n_ss + ss0;
-                        bulk_g2s(dst, src_base + tile0 * bytes_per_step, cnt * bytes_per_step, full);
+                    const uint32_t stage_base = smem_u32(smem + S::oStages + stage * S::kStageBytes);
+                    const uint8_t* src = op.store + ((long long)rp * op.n_kb + kb0) * op.blob_stride;
+                    if (contiguous) {
+                        if (lane == 0) bulk_g2s(stage_base, src, nb * op.blob_read, full);
+                    } else if (lane < nb) {
+                        bulk_g2s(stage_base + lane * op.blob_read, src + (long long)lane * op.blob_stride, op.blob_read, full);
                     }
                     if (++stage == S::kStages) { stage = 0; wraps++; }
                     if (++rp == op.n_rp) { rp = 0; ch++; new_chunk = true; }
@@ -463,8 +454,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 if (op.phase > 0) phase_known = op.phase - 1;          // (meaningless after an abort; unused then)
                 if (go == 0) { stop = true; break; }
                 if (go == 1) {
-                    const int ss0 = ch * op.chunk_steps;
-                    const int cnt = min(op.chunk_steps, op.n_ss - ss0);
+                    const int ss0 = ch * op.chunk_blobs * kBlobSteps;
+                    const int cnt = min(op.chunk_blobs, op.n_kb - ch * op.chunk_blobs) * kBlobSteps;
                     int* xsum = reinterpret_cast<int*>(xs + S::kXsumOff);
                     float* xscale = reinterpret_cast<float*>(xs + S::kXscaleOff);
                     const int n_items = cnt * op.batch;                // item = (batch row, superstep)
@@ -573,13 +564,13 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     stop = true;
                     break;
                 }
-                struct { int ch, rp, cnt, n_tiles, seg, n_out, n_chunks, bits, n_fields, phase, zero_adjust, batch;
+                struct { int ch, rp, cnt, seg, n_out, n_chunks, blob_read, n_fields, phase, zero_adjust, batch;
                          uint16_t* y; float* partial; unsigned* tile_count; uint8_t width[8], shift[8]; } d;
                 {
                     const UnitDesc ud = *(reinterpret_cast<const UnitDesc*>(smem + S::oDesc) + stage);
                     const GemvOp& od = *reinterpret_cast<const GemvOp*>(opring + ud.op_slot * S::kOpBytes);
-                    d.ch = ud.ch; d.rp = ud.rp; d.cnt = ud.cnt; d.n_tiles = ud.n_tiles; d.seg = ud.seg;
-                    d.n_out = od.n_out; d.n_chunks = od.n_chunks; d.bits = od.bits; d.n_fields = od.n_fields;
+                    d.ch = ud.ch; d.rp = ud.rp; d.cnt = ud.nb * kBlobSteps; d.seg = ud.seg;
+                    d.n_out = od.n_out; d.n_chunks = od.n_chunks; d.blob_read = od.blob_read; d.n_fields = od.n_fields;
                     d.phase = od.phase; d.zero_adjust = od.zero_adjust; d.batch = od.batch;
                     d.y = od.y; d.partial = od.partial; d.tile_count = od.tile_count;
 #pragma unroll
@@ -594,7 +585,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 __syncwarp();
                 const bool live = !flags[0];
                 const int B = d.batch;
-                const bool two_tiles = d.n_tiles > 1, two_pass = MAXB > 1 && B > 4;
+                const bool two_tiles = true, two_pass = MAXB > 1 && B > 4;
                 const uint8_t* xs = smem + S::oX + slot * S::kXSlotBytes;
 
                 float tot[2][NP][2];
@@ -619,25 +610,25 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     }
                     const int* xsum = reinterpret_cast<const int*>(xs + S::kXsumOff);
                     const float* xscale = reinterpret_cast<const float*>(xs + S::kXscaleOff);
-                    const int tile_code_bytes = d.cnt * 512;                       // per unit of field width
-                    const uint32_t* meta_s = reinterpret_cast<const uint32_t*>(st + d.n_tiles * d.cnt * 512 * d.bits);
-
                     for (int s = 0; s < d.cnt; s++) {
+                        const uint8_t* blob = st + (s / kBlobSteps) * d.blob_read;       // this superstep's blob (prefix)
+                        const int ssl = s % kBlobSteps;
+                        const uint32_t* meta_s = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, 0));
                         int v[2][2][2][2];
 #pragma unroll
                         for (int i = 0; i < 16; i++) (&v[0][0][0][0])[i] = 0;
-                        const uint8_t* fs = st;
+                        int prefix = 0;
                         for (int fi = 0; fi < d.n_fields; fi++) {
                             const int f = d.width[fi];
-                            const uint8_t* f0 = fs + s * f * 512;
-                            const uint8_t* f1 = f0 + tile_code_bytes * f;
+                            const uint8_t* f0 = blob + blob_field_off(prefix, f, ssl, 0);
+                            const uint8_t* f1 = f0 + f * 512;
                             switch (f) {
                                 case 8: field_step<8, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
                                 case 4: field_step<4, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
                                 case 2: field_step<2, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
                                 default: field_step<1, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
                             }
-                            fs += d.n_tiles * tile_code_bytes * f;
+                            prefix += f;
                         }
                         // group epilogue: y += s * 2^-e * (v - z * sum x_int)
 #pragma unroll
@@ -645,12 +636,12 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                             if (tile == 1 && !two_tiles) break;
 #pragma unroll
                             for (int grp = 0; grp < 2; grp++) {
-                                const uint32_t m0 = meta_s[(tile * d.cnt + s) * 32 + grp * 16 + g];
-                                const uint32_t m1 = meta_s[(tile * d.cnt + s) * 32 + grp * 16 + g + 8];
+                                const uint32_t m0 = meta_s[tile * 32 + grp * 16 + g];
+                                const uint32_t m1 = meta_s[tile * 32 + grp * 16 + g + 8];
                                 const float s0 = __half2float(__ushort_as_half((unsigned short)(m0 & 0xffffu)));
                                 const float s1 = __half2float(__ushort_as_half((unsigned short)(m1 & 0xffffu)));
-                                const int z0 = __half2int_rn(__ushort_as_half((unsigned short)(m0 >> 16))) - d.zero_adjust;
-                                const int z1 = __half2int_rn(__ushort_as_half((unsigned short)(m1 >> 16))) - d.zero_adjust;
+                                const int z0 = (int)(m0 >> 16) - d.zero_adjust;
+                                const int z1 = (int)(m1 >> 16) - d.zero_adjust;
 #pragma unroll
                                 for (int p = 0; p < NP; p++) {
                                     // batch 1: only the class-0 lane subtracts the zero-point term

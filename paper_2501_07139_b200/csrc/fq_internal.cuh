@@ -12,8 +12,7 @@ namespace fq {
 // One stored variant of a layer.
 struct Variant {
     bool present = false;
-    void* codes = nullptr;       // field arrays, concatenated, most significant first
-    void* meta = nullptr;        // [row_tile][group][16] (scale, zero) words
+    void* store = nullptr;       // blobs: scale/zero words + field arrays (fq_layout.cuh)
 };
 
 struct Layer {
@@ -27,21 +26,22 @@ constexpr int kUnitRowTiles = 2;   // a decode unit covers two 16-row tiles (32 
 
 // What one decode op needs on the device.
 struct GemvOp {
-    const uint8_t* field_ptr[kMaxFields];
+    const uint8_t* store;        // blobs [row_pair][k_blob]
+    int blob_stride;             // bytes from one blob to the next (size of the stored variant's blobs)
+    int blob_read;               // bytes of every blob that this op reads (all of it, or a nested child's prefix)
     uint8_t field_width[kMaxFields];
     uint8_t field_shift[kMaxFields];
     int n_fields;
     int bits;                    // code bytes per tile superstep = 512 * bits
-    const uint32_t* meta;
     const uint16_t* x;           // fp16 [batch][k_in]
     uint16_t* y;                 // fp16 [batch][n_out]
     float* partial;              // split-K partial sums (unused when n_chunks == 1)
     unsigned* tile_count;        // split-K arrival counters, one per row pair
     int n_out, k_in;
-    int n_rt, n_ss;              // row tiles, supersteps
+    int n_ss, n_kb;              // supersteps, k blobs
     int n_rp;                    // row pairs = units per K chunk
     int n_chunks;                // K chunks
-    int chunk_steps;             // supersteps per K chunk (the last chunk may be shorter)
+    int chunk_blobs;             // k blobs per K chunk (the last chunk may be shorter)
     int batch;
     int zero_adjust;             // subtracted from every zero point (mid-point fill of a nested child)
     int phase;                   // -1: no ordering
@@ -80,15 +80,16 @@ int ensure_workspace(Ctx* ctx, size_t bytes);
 int launch_quantize(const float* w, int n_out, int k_in, int bits, uint8_t* codes, uint16_t* scales,
                     uint16_t* zeros, cudaStream_t st);
 int launch_pack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int n_out, int k_in,
-                const FieldList& fl, void* code_out, void* meta_out, cudaStream_t st);
-int launch_export_packed(const void* codes, int n_out, int k_in, int bits, const FieldList& fl,
+                int stored_bits, const FieldList& fl, void* store, cudaStream_t st);
+int launch_export_packed(const void* store, int n_out, int k_in, int bits, const FieldList& fl,
                          uint32_t* out, cudaStream_t st);
-int launch_export_planes(const void* codes, int n_out, int k_in, int bits, const FieldList& fl,
+int launch_export_planes(const void* store, int n_out, int k_in, int bits, const FieldList& fl,
                          uint32_t* out, cudaStream_t st);
-int launch_export_meta(const void* meta, int n_out, int k_in, uint16_t* scales, uint16_t* zeros, cudaStream_t st);
+int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, uint16_t* scales, uint16_t* zeros,
+                       cudaStream_t st);
 
-// Chunking policy of the decode kernel: supersteps (256 columns) per K chunk.
-int gemv_chunk_steps(int bits, int batch);
+// Chunking policy of the decode kernel: k blobs (512 columns) per K chunk.
+int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_floats_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
 int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st);

@@ -5,8 +5,14 @@
 //   PACKED b bits : the binary decomposition of b   (7 -> 4,2,1;  5 -> 4,1;  3 -> 2,1 ...)
 //   PLANES parent : a 2-bit top field (bits 7,6) followed by six 1-bit planes (5 .. 0),
 //                   so a b-bit child is the first b-1 arrays = the first b/8 of the bytes.
-// Every array is tiled: tile = 16 rows x 256 columns ("superstep"), tiles ordered
-// [row_tile][superstep], and inside a tile  [f chunks][32 lanes][16 bytes].
+// Storage is cut into BLOBS: one blob = one row pair (32 rows = two 16-row tiles) x 512 columns
+// (two "supersteps" of 256).  A blob holds, in this order,
+//     scale/zero words   [superstep][tile][group][16 rows]                       (512 B)
+//     field array 0      [superstep][tile][f0 chunks][32 lanes][16 B]            (2048 * f0 B)
+//     field array 1 ...                                                          (most significant first)
+// and blobs are ordered [row_pair][k_blob].  Everything a decode unit needs is therefore ONE
+// contiguous range for a PACKED variant (one bulk copy), and for a nested child the first
+// 512 + 2048*b bytes of every blob (one bulk copy per blob): lower planes are never touched.
 // The order inside a tile is the order in which a warp consumes the values as A-operand
 // registers of the 8-bit mma.m16n8k32 (lane = 4*g + c owns rows g, g+8; in k32 step j it owns
 // columns 32j + 4c .. +3 and 32j + 16 + 4c .. +3).  A 32-bit word holds P = 8/f A-registers
@@ -15,7 +21,7 @@
 // register of k32 step  j = P*chunk + t  (values scaled by 2^(t*f)), with no shift at all;
 // the four words of a lane's 16-byte chunk are the four A registers a0..a3.
 //
-// Metadata: [row_tile][group][16 rows] words, low half = scale, high half = zero (fp16).
+// Scale/zero word: low half = fp16 scale, high half = the zero point as an unsigned integer.
 #pragma once
 #include <cstdint>
 
@@ -71,10 +77,22 @@ FQ_HD int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 FQ_HD int row_tiles(int n_out) { return (n_out + kTileRows - 1) / kTileRows; }
 FQ_HD int supersteps(int k_in) { return (k_in + kStepCols - 1) / kStepCols; }
 
-// Bytes of one field array.
-FQ_HD int64_t field_bytes(int n_out, int k_in, int f)
+constexpr int kBlobSteps = 2;             // supersteps per blob
+constexpr int kBlobTiles = 2;             // row tiles per blob (a row pair)
+constexpr int kBlobMetaBytes = kBlobSteps * kBlobTiles * 128;
+
+FQ_HD int row_pairs(int n_out) { return (row_tiles(n_out) + kBlobTiles - 1) / kBlobTiles; }
+FQ_HD int k_blobs(int k_in) { return (supersteps(k_in) + kBlobSteps - 1) / kBlobSteps; }
+// Bytes of a blob whose fields add up to `bits` bits (also: prefix of a nested parent's blob that a
+// `bits`-bit child reads).
+FQ_HD int blob_bytes(int bits) { return kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * bits; }
+FQ_HD int64_t store_bytes(int n_out, int k_in, int bits) { return (int64_t)row_pairs(n_out) * k_blobs(k_in) * blob_bytes(bits); }
+// Offsets inside a blob: scale/zero words of (superstep ssl, tile), and the tile of field width f
+// that comes after fields adding up to prefix_bits.
+FQ_HD int blob_meta_off(int ssl, int tile) { return (ssl * kBlobTiles + tile) * 128; }
+FQ_HD int blob_field_off(int prefix_bits, int f, int ssl, int tile)
 {
-    return (int64_t)row_tiles(n_out) * supersteps(k_in) * f * 512;
+    return kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * prefix_bits + (ssl * kBlobTiles + tile) * f * 512;
 }
 
 // Position of the field of element (row r in 0..15, column kk in 0..255) inside a tile of a

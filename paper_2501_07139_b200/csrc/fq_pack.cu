@@ -91,59 +91,60 @@ int launch_quantize(const float* w, int n_out, int k_in, int bits, uint8_t* code
 }
 
 // ---------------------------------------------------------------------------------------
-// Packer: one thread per 32-bit word of a field array (gathers 32/f codes).
+// Packer: one thread per 32-bit word of the stored variant (blob layout, see fq_layout.cuh).
 // ---------------------------------------------------------------------------------------
-struct PackArgs {
-    const uint8_t* codes;
-    int n_out, k_in, n_ss;
-    FieldList fl;
-    long long field_word_base[kMaxFields + 1];   // first word of every field array, cumulative
-    uint32_t* out;
+struct StoreArgs {
+    const uint8_t* codes;          // pack: canonical codes, one per byte
+    const uint16_t* scales;
+    const uint16_t* zeros;
+    uint32_t* store;               // the stored variant
+    int n_out, k_in, n_kb, groups;
+    int stored_bits;               // bits of the stored variant (size of its blobs)
+    FieldList fl;                  // fields that are written / read
+    long long total_words;
 };
 
-__global__ void __launch_bounds__(256) pack_kernel(const PackArgs a)
+__global__ void __launch_bounds__(256) pack_kernel(const StoreArgs a)
 {
-    const long long total = a.field_word_base[a.fl.n];
-    for (long long wi = (long long)blockIdx.x * blockDim.x + threadIdx.x; wi < total;
+    const int blob_words = blob_bytes(a.stored_bits) / 4;
+    for (long long wi = (long long)blockIdx.x * blockDim.x + threadIdx.x; wi < a.total_words;
          wi += (long long)gridDim.x * blockDim.x) {
-        int fi = 0;
-        while (wi >= a.field_word_base[fi + 1]) fi++;
-        const int f = a.fl.width[fi], sh = a.fl.shift[fi];
-        const long long local = wi - a.field_word_base[fi];
-        const int words_per_tile = f * 128;                    // f chunks * 32 lanes * 4 words
-        const long long tile = local / words_per_tile;
-        const int in_tile = (int)(local % words_per_tile);
-        const int chunk = in_tile >> 7, lane = (in_tile >> 2) & 31, word = in_tile & 3;
-        const int rt = (int)(tile / a.n_ss), ss = (int)(tile % a.n_ss);
-        const unsigned mask = (1u << f) - 1u;
+        const long long blob = wi / blob_words;
+        const int off = (int)(wi % blob_words) * 4;               // byte offset inside the blob
+        const int rp = (int)(blob / a.n_kb), kb = (int)(blob % a.n_kb);
         unsigned v = 0;
-        for (int q = 0; q < 32 / f; q++) {
-            int r, kk, bit;
-            field_owner(f, chunk, lane, word, q, r, kk, bit);
-            const long long n = (long long)rt * kTileRows + r;
-            const long long k = (long long)ss * kStepCols + kk;
-            unsigned code = 0;
-            if (n < a.n_out && k < a.k_in) code = a.codes[n * a.k_in + k];
-            v |= ((code >> sh) & mask) << bit;
+        if (off < kBlobMetaBytes) {
+            // scale/zero word: [superstep][tile][group][16 rows]
+            const int r = (off >> 2) & 15, grp = (off >> 6) & 1, tile = (off >> 7) & 1, ssl = off >> 8;
+            const long long n = ((long long)rp * kBlobTiles + tile) * kTileRows + r;
+            const int g = (kb * kBlobSteps + ssl) * 2 + grp;
+            if (n < a.n_out && g < a.groups) {
+                const float z = __half2float(__ushort_as_half(a.zeros[n * a.groups + g]));
+                const unsigned zi = (unsigned)fminf(fmaxf(rintf(z), 0.f), 65535.f);
+                v = (unsigned)a.scales[n * a.groups + g] | (zi << 16);
+            }
+        } else {
+            int rem = off - kBlobMetaBytes, fi = 0;
+            while (rem >= kBlobSteps * kBlobTiles * 512 * a.fl.width[fi]) {
+                rem -= kBlobSteps * kBlobTiles * 512 * a.fl.width[fi];
+                fi++;
+            }
+            const int f = a.fl.width[fi], sh = a.fl.shift[fi];
+            const int st = rem / (f * 512), in_tile = rem % (f * 512);       // st = ssl * 2 + tile
+            const int ssl = st / kBlobTiles, tile = st % kBlobTiles;
+            const int chunk = in_tile >> 9, lane = (in_tile >> 4) & 31, word = (in_tile >> 2) & 3;
+            const unsigned mask = (1u << f) - 1u;
+            for (int q = 0; q < 32 / f; q++) {
+                int r, kk, bit;
+                field_owner(f, chunk, lane, word, q, r, kk, bit);
+                const long long n = ((long long)rp * kBlobTiles + tile) * kTileRows + r;
+                const long long k = ((long long)kb * kBlobSteps + ssl) * kStepCols + kk;
+                unsigned code = 0;
+                if (n < a.n_out && k < a.k_in) code = a.codes[n * a.k_in + k];
+                v |= ((code >> sh) & mask) << bit;
+            }
         }
-        a.out[wi] = v;
-    }
-}
-
-// Metadata: [row_tile][group (padded to 2 per superstep)][16 rows] words (scale | zero << 16).
-__global__ void __launch_bounds__(256)
-pack_meta_kernel(const uint16_t* __restrict__ scales, const uint16_t* __restrict__ zeros, int n_out, int groups,
-                 int groups_padded, long long total, uint32_t* __restrict__ out)
-{
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const int r = (int)(i & 15);
-        const long long tg = i >> 4;
-        const int g = (int)(tg % groups_padded);
-        const long long n = (tg / groups_padded) * kTileRows + r;
-        uint32_t v = 0;
-        if (n < n_out && g < groups) v = (uint32_t)scales[n * groups + g] | ((uint32_t)zeros[n * groups + g] << 16);
-        out[i] = v;
+        a.store[wi] = v;
     }
 }
 
@@ -155,50 +156,53 @@ static unsigned grid_for(long long total)
 }
 
 int launch_pack(const uint8_t* codes, const uint16_t* scales, const uint16_t* zeros, int n_out, int k_in,
-                const FieldList& fl, void* code_out, void* meta_out, cudaStream_t st)
+                int stored_bits, const FieldList& fl, void* store, cudaStream_t st)
 {
-    PackArgs a{};
-    a.codes = codes; a.n_out = n_out; a.k_in = k_in; a.n_ss = supersteps(k_in); a.fl = fl;
-    a.out = (uint32_t*)code_out;
-    long long base = 0;
-    for (int i = 0; i < fl.n; i++) {
-        a.field_word_base[i] = base;
-        base += field_bytes(n_out, k_in, fl.width[i]) / 4;
-    }
-    a.field_word_base[fl.n] = base;
-    pack_kernel<<<grid_for(base), 256, 0, st>>>(a);
-    FQ_CUDA_OK(cudaGetLastError());
-    const int groups = k_in / kGroup, groups_padded = supersteps(k_in) * 2;
-    const long long total = (long long)row_tiles(n_out) * groups_padded * 16;
-    pack_meta_kernel<<<grid_for(total), 256, 0, st>>>(scales, zeros, n_out, groups, groups_padded, total,
-                                                    (uint32_t*)meta_out);
+    StoreArgs a{};
+    a.codes = codes; a.scales = scales; a.zeros = zeros; a.store = (uint32_t*)store;
+    a.n_out = n_out; a.k_in = k_in; a.n_kb = k_blobs(k_in); a.groups = k_in / kGroup;
+    a.stored_bits = stored_bits; a.fl = fl;
+    a.total_words = store_bytes(n_out, k_in, stored_bits) / 4;
+    pack_kernel<<<grid_for(a.total_words), 256, 0, st>>>(a);
     FQ_CUDA_OK(cudaGetLastError());
     return FQ_OK;
 }
 
 // ---------------------------------------------------------------------------------------
-// Exporters: rebuild canonical bytes from the field arrays (test / reporting support).
+// Exporters: rebuild canonical bytes from the stored variant (test / reporting support).
 // ---------------------------------------------------------------------------------------
 struct ExportArgs {
-    const uint8_t* field_ptr[kMaxFields];
-    FieldList fl;
-    int n_out, k_in, n_ss, bits;
+    const uint8_t* store;
+    FieldList fl;                  // fields to read (a prefix of the stored ones for a nested child)
+    int n_out, k_in, n_kb, groups, stored_bits, bits;
     uint32_t* out;
+    uint16_t* scales;
+    uint16_t* zeros;
     long long total_words;
 };
 
-// Bits [lo_shift .. ] of the stored code of element (n, k), assembled from the field arrays.
+__device__ __forceinline__ const uint8_t* blob_of(const ExportArgs& a, long long n, long long k, int& tile, int& ssl)
+{
+    const int rt = (int)(n / kTileRows), ss = (int)(k / kStepCols);
+    tile = rt % kBlobTiles;
+    ssl = ss % kBlobSteps;
+    return a.store + ((long long)(rt / kBlobTiles) * a.n_kb + ss / kBlobSteps) * blob_bytes(a.stored_bits);
+}
+
+// The stored code of element (n, k), assembled from the fields in a.fl (shifts as stored).
 __device__ __forceinline__ unsigned stored_code(const ExportArgs& a, long long n, long long k)
 {
-    const int rt = (int)(n / kTileRows), r = (int)(n % kTileRows);
-    const int ss = (int)(k / kStepCols), kk = (int)(k % kStepCols);
+    int tile, ssl;
+    const uint8_t* blob = blob_of(a, n, k, tile, ssl);
+    const int r = (int)(n % kTileRows), kk = (int)(k % kStepCols);
     unsigned code = 0;
+    int prefix = 0;
     for (int fi = 0; fi < a.fl.n; fi++) {
         const int f = a.fl.width[fi];
         const FieldPos p = field_pos(f, r, kk);
-        const long long tile = (long long)rt * a.n_ss + ss;
-        const uint32_t wv = *reinterpret_cast<const uint32_t*>(a.field_ptr[fi] + tile * (f * 512) + p.word_byte);
+        const uint32_t wv = *reinterpret_cast<const uint32_t*>(blob + blob_field_off(prefix, f, ssl, tile) + p.word_byte);
         code |= ((wv >> p.bit) & ((1u << f) - 1u)) << a.fl.shift[fi];
+        prefix += f;
     }
     return code;
 }
@@ -237,58 +241,59 @@ __global__ void __launch_bounds__(256) export_planes_kernel(const ExportArgs a)
     }
 }
 
-static void fill_export(ExportArgs& a, const void* codes, int n_out, int k_in, int bits, const FieldList& fl,
-                        uint32_t* out)
+__global__ void __launch_bounds__(256) export_meta_kernel(const ExportArgs a)
 {
-    a.fl = fl; a.n_out = n_out; a.k_in = k_in; a.n_ss = supersteps(k_in); a.bits = bits; a.out = out;
-    const uint8_t* p = (const uint8_t*)codes;
-    for (int i = 0; i < fl.n; i++) {
-        a.field_ptr[i] = p;
-        p += field_bytes(n_out, k_in, fl.width[i]);
+    const long long total = (long long)a.n_out * a.groups;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long n = i / a.groups;
+        const int g = (int)(i % a.groups);
+        int tile, ssl;
+        const uint8_t* blob = blob_of(a, n, (long long)g * kGroup, tile, ssl);
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile) + (g & 1) * 64 +
+                                                              (int)(n % kTileRows) * 4);
+        a.scales[i] = (uint16_t)(v & 0xffffu);
+        a.zeros[i] = __half_as_ushort(__float2half_rn((float)(v >> 16)));
     }
+}
+
+static void fill_export(ExportArgs& a, const void* store, int n_out, int k_in, int stored_bits, int bits,
+                        const FieldList& fl)
+{
+    a.store = (const uint8_t*)store; a.fl = fl; a.n_out = n_out; a.k_in = k_in; a.n_kb = k_blobs(k_in);
+    a.groups = k_in / kGroup; a.stored_bits = stored_bits; a.bits = bits;
     a.total_words = (long long)n_out * k_in * bits / 32;
 }
 
-int launch_export_packed(const void* codes, int n_out, int k_in, int bits, const FieldList& fl, uint32_t* out,
+int launch_export_packed(const void* store, int n_out, int k_in, int bits, const FieldList& fl, uint32_t* out,
                          cudaStream_t st)
 {
     ExportArgs a{};
-    fill_export(a, codes, n_out, k_in, bits, fl, out);
+    fill_export(a, store, n_out, k_in, bits, bits, fl);
+    a.out = out;
     export_packed_kernel<<<grid_for(a.total_words), 256, 0, st>>>(a);
     FQ_CUDA_OK(cudaGetLastError());
     return FQ_OK;
 }
 
-int launch_export_planes(const void* codes, int n_out, int k_in, int bits, const FieldList& fl, uint32_t* out,
+int launch_export_planes(const void* store, int n_out, int k_in, int bits, const FieldList& fl, uint32_t* out,
                          cudaStream_t st)
 {
     ExportArgs a{};
-    fill_export(a, codes, n_out, k_in, bits, fl, out);
+    fill_export(a, store, n_out, k_in, 8, bits, fl);
+    a.out = out;
     export_planes_kernel<<<grid_for(a.total_words), 256, 0, st>>>(a);
     FQ_CUDA_OK(cudaGetLastError());
     return FQ_OK;
 }
 
-__global__ void __launch_bounds__(256)
-export_meta_kernel(const uint32_t* __restrict__ meta, int n_out, int groups, int groups_padded,
-                   uint16_t* __restrict__ scales, uint16_t* __restrict__ zeros)
+int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, uint16_t* scales, uint16_t* zeros,
+                       cudaStream_t st)
 {
-    const long long total = (long long)n_out * groups;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const long long n = i / groups;
-        const int g = (int)(i % groups);
-        const uint32_t v = meta[((n / kTileRows) * groups_padded + g) * 16 + (n % kTileRows)];
-        scales[i] = (uint16_t)(v & 0xffffu);
-        zeros[i] = (uint16_t)(v >> 16);
-    }
-}
-
-int launch_export_meta(const void* meta, int n_out, int k_in, uint16_t* scales, uint16_t* zeros, cudaStream_t st)
-{
-    const int groups = k_in / kGroup;
-    export_meta_kernel<<<grid_for((long long)n_out * groups), 256, 0, st>>>(
-        (const uint32_t*)meta, n_out, groups, supersteps(k_in) * 2, scales, zeros);
+    ExportArgs a{};
+    fill_export(a, store, n_out, k_in, stored_bits, stored_bits, FieldList{});
+    a.scales = scales; a.zeros = zeros;
+    export_meta_kernel<<<grid_for((long long)n_out * a.groups), 256, 0, st>>>(a);
     FQ_CUDA_OK(cudaGetLastError());
     return FQ_OK;
 }

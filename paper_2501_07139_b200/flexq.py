@@ -20,7 +20,7 @@ _LIB_PATH = os.path.join(_HERE, "libflexq.so")
 _lib = None
 
 EXPORTS = [
-    "fq_create", "fq_destroy", "fq_code_bytes", "fq_meta_bytes", "fq_quantize_layer", "fq_pack_layer",
+    "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
     "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static",
 ]
@@ -48,12 +48,10 @@ def lib():
     vp, i, u64 = C.c_void_p, C.c_int, C.c_uint64
     L.fq_create.argtypes = [C.POINTER(vp), i, i]
     L.fq_destroy.argtypes = [vp]
-    L.fq_code_bytes.argtypes = [i, i, i, i]
-    L.fq_code_bytes.restype = C.c_size_t
-    L.fq_meta_bytes.argtypes = [i, i, i]
-    L.fq_meta_bytes.restype = C.c_size_t
+    L.fq_store_bytes.argtypes = [i, i, i, i]
+    L.fq_store_bytes.restype = C.c_size_t
     L.fq_quantize_layer.argtypes = [vp, i, i, i, i, vp, vp, vp, vp]
-    L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp]
+    L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
     L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
     L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
@@ -80,12 +78,8 @@ def fq_strerror(code: int) -> str:
     return lib().fq_strerror(int(code)).decode()
 
 
-def fq_code_bytes(n_out: int, k_in: int, bits: int, fmt: int) -> int:
-    return int(lib().fq_code_bytes(n_out, k_in, bits, fmt))
-
-
-def fq_meta_bytes(n_out: int, k_in: int, group: int = 128) -> int:
-    return int(lib().fq_meta_bytes(n_out, k_in, group))
+def fq_store_bytes(n_out: int, k_in: int, bits: int, fmt: int) -> int:
+    return int(lib().fq_store_bytes(n_out, k_in, bits, fmt))
 
 
 def _stream() -> int:
@@ -112,14 +106,14 @@ def fq_quantize_layer(w: torch.Tensor, bits: int, group: int = 128):
 
 
 class FlexQ:
-    """One library context.  Keeps the retained device buffers (codes, metadata) alive."""
+    """One library context.  Keeps the retained device buffers (the stored variants) alive."""
 
     def __init__(self, n_layers: int, device: int = 0):
         self._h = C.c_void_p()
         self.device = torch.device("cuda", device)
         _check(lib().fq_create(C.byref(self._h), device, n_layers), "fq_create")
         self.n_layers = n_layers
-        self._keep = {}          # (layer, bits) -> (codes, meta) tensors retained by the context
+        self._keep = {}          # (layer, bits) -> stored variant retained by the context
         self._stack_keep = None
 
     # -- lifetime -----------------------------------------------------------------
@@ -141,19 +135,17 @@ class FlexQ:
         assert codes.is_cuda and codes.dtype == torch.uint8 and codes.is_contiguous()
         assert scales.dtype == torch.float16 and zeros.dtype == torch.float16
         n, k = codes.shape
-        cb, mb = fq_code_bytes(n, k, bits, fmt), fq_meta_bytes(n, k, group)
-        if cb == 0 or mb == 0:
+        sb = fq_store_bytes(n, k, bits, fmt)
+        if sb == 0 or group != 128:
             # let the library name the problem
             _check(lib().fq_pack_layer(self._h, layer, n, k, bits, group, fmt, codes.data_ptr(), scales.data_ptr(),
-                                       zeros.data_ptr(), codes.data_ptr(), codes.data_ptr(), _stream()),
-                   "fq_pack_layer")
-        code_out = torch.empty(cb, dtype=torch.uint8, device=self.device)
-        meta_out = torch.empty(mb, dtype=torch.uint8, device=self.device)
+                                       zeros.data_ptr(), codes.data_ptr(), _stream()), "fq_pack_layer")
+        store = torch.empty(sb, dtype=torch.uint8, device=self.device)
         _check(lib().fq_pack_layer(self._h, layer, n, k, bits, group, fmt, codes.data_ptr(),
                                    scales.contiguous().data_ptr(), zeros.contiguous().data_ptr(),
-                                   code_out.data_ptr(), meta_out.data_ptr(), _stream()), "fq_pack_layer")
-        self._keep[(layer, bits)] = (code_out, meta_out)
-        return code_out, meta_out
+                                   store.data_ptr(), _stream()), "fq_pack_layer")
+        self._keep[(layer, bits)] = store
+        return store
 
     # -- configuration -------------------------------------------------------------------
     def fq_set_config(self, bits: Sequence[int]) -> int:

@@ -30,14 +30,13 @@ def test_every_declared_symbol_is_exported():
 
 def test_size_helpers_and_error_strings_need_no_gpu():
     import paper_2501_07139_b200 as P
-    assert P.fq_code_bytes(4096, 4096, 4, P.FQ_FMT_PACKED) == 8_388_608
-    assert P.fq_code_bytes(4096, 4096, 8, P.FQ_FMT_PLANES) == 16_777_216
-    assert P.fq_code_bytes(17, 128, 3, P.FQ_FMT_PACKED) == 2 * 1 * 512 * 3        # padded to 32 rows x 256 cols
-    assert P.fq_code_bytes(16, 100, 4, P.FQ_FMT_PACKED) == 0
-    assert P.fq_code_bytes(16, 128, 9, P.FQ_FMT_PACKED) == 0
-    assert P.fq_code_bytes(16, 128, 4, P.FQ_FMT_PLANES) == 0
-    assert P.fq_meta_bytes(4096, 4096) == 524_288
-    assert P.fq_meta_bytes(16, 128, 64) == 0
+    assert P.fq_store_bytes(4096, 4096, 4, P.FQ_FMT_PACKED) == 8_388_608 + 524_288     # codes + scale/zero words
+    assert P.fq_store_bytes(4096, 4096, 8, P.FQ_FMT_PLANES) == 16_777_216 + 524_288
+    assert P.fq_store_bytes(17, 128, 3, P.FQ_FMT_PACKED) == 512 + 2048 * 3                # one blob: 32 rows x 512 cols
+    assert P.fq_store_bytes(33, 1024, 5, P.FQ_FMT_PACKED) == 2 * 2 * (512 + 2048 * 5)
+    assert P.fq_store_bytes(16, 100, 4, P.FQ_FMT_PACKED) == 0
+    assert P.fq_store_bytes(16, 128, 9, P.FQ_FMT_PACKED) == 0
+    assert P.fq_store_bytes(16, 128, 4, P.FQ_FMT_PLANES) == 0
     for code in range(0, -10, -1):
         assert P.fq_strerror(code) != "unknown error"
     assert P.fq_strerror(-99) == "unknown error"

@@ -54,7 +54,7 @@ def test_pack_export_planes_bit_exact_and_nested(P, shape):
     n, k = shape
     q8, s, z = make_layer(92, 0, n, k, 8)
     fq = P.FlexQ(1)
-    code_buf, _ = fq.fq_pack_layer(0, *to_dev(q8, s, z), 8, P.FQ_FMT_PLANES)
+    code_buf = fq.fq_pack_layer(0, *to_dev(q8, s, z), 8, P.FQ_FMT_PLANES)
     before = code_buf.clone()
     ref = O.pack_planes(q8)
     for b in range(2, 9):
