@@ -32,7 +32,7 @@ namespace fq {
 #define FQ_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return FQ_ERR_CUDA; } while (0)
 
 #ifndef FQ_GEMV_WARPS
-#define FQ_GEMV_WARPS 8
+#define FQ_GEMV_WARPS 10
 #endif
 #ifndef FQ_GEMV_UNIT_BYTES
 #define FQ_GEMV_UNIT_BYTES 17408
@@ -84,7 +84,7 @@ template <int MAXB> struct GemvSmem {
     static constexpr int oReleased = oBars + 2 * kStages * 8;        // u32[S]: uses of a stage that were released
     static constexpr int oCtl = oReleased + kStages * 4;             // x_ready[XS], x_pending[XS], flags[2]
     static constexpr int kTotal = oCtl + 64;
-    static_assert(kStages >= kConsumerWarps, "decode kernel: ring shorter than the number of consumers");
+    static_assert(kStages >= 4, "decode kernel: no room for a ring");
     static_assert(kTotal <= 232448, "decode kernel: shared memory over the 227 KB per-CTA limit");
 };
 
@@ -161,6 +161,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Counter updates that carry their own ordering instead of a separate membar: the release half makes
+// this warp's earlier stores (ordered before it by __syncwarp) visible first, the acquire half orders
+// the loads that follow.
+__device__ __forceinline__ unsigned atom_add_acq_rel_u32(unsigned* p, unsigned v)
+{
+    unsigned old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void red_add_release_u64(unsigned long long* p, unsigned long long v)
+{
+    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p)
 {
@@ -708,14 +721,12 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                                 if (MAXB == 1) { if (c == 0) pu[lr] = tot[tile][0][r]; }
                                 else pu[lr * BW + 4 * p + c] = tot[tile][p][r];
                             }
-                    __threadfence();
                     __syncwarp();
                     unsigned old = 0;
-                    if (lane == 0) old = atomicAdd(d.tile_count + d.rp, 1u);
+                    if (lane == 0) old = atom_add_acq_rel_u32(d.tile_count + d.rp, 1u);
                     old = __shfl_sync(0xffffffffu, old, 0);
                     wrote_final = false;
                     if (old == (unsigned)(d.n_chunks - 1)) {
-                        __threadfence();
                         const float* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW);
                         for (int e = lane; e < 32 * BW; e += 32) {   // e = local row * BW + batch entry
                             float sum = 0.f;
@@ -728,9 +739,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     }
                 }
                 if (d.phase >= 0) {
-                    if (wrote_final) __threadfence();                // y must be visible before the phase count moves
-                    __syncwarp();
-                    if (lane == 0) atomicAdd(sa.phase_done + d.phase, 1ull);
+                    __syncwarp();                                    // y is ordered before the release below
+                    if (lane == 0) red_add_release_u64(sa.phase_done + d.phase, 1ull);
                 }
             }
         }
