@@ -145,7 +145,10 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host,
 /* Prefill / calibration-set evaluation (Sec. III-B: every candidate EQM is run forward over
  * token sequences):  Y[m][n] = sum_k X[m][k] * w^[n][k].
  *   X_dev bf16 [M][ldx >= k_in], Y_dev bf16 [M][ldy >= n_out], row-major, 16-byte aligned,
- *   ldx and ldy multiples of 8.  Tensor-core path, fp32 accumulation. */
+ *   ldx and ldy multiples of 8, 1 <= M <= 2^20.  The layer is dequantised to bf16 (one rounding of
+ *   the exact (q - z) * s) into a workspace of n_out*k_in*2 bytes that the context owns (grown with
+ *   a device allocation when a larger layer is first used), then multiplied on the tensor cores
+ *   (tcgen05, fp32 accumulation in TMEM).  Enqueues two kernels on `stream`. */
 int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx,
             uint16_t* Y_dev, int ldy, void* stream);
 

@@ -166,6 +166,7 @@ int fq_destroy(fq_ctx* ctx)
         if (ctx->status_dev) cudaFree(ctx->status_dev);
         if (ctx->stack_dev) cudaFree(ctx->stack_dev);
         if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
+        if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
     }
     delete ctx;
     return FQ_OK;
@@ -348,6 +349,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
     if (!(ctx->stack_valid && ctx->stack_key == key)) {
         if (ctx->stack_host_bytes < hdr_off + sizeof(StackHeader)) {
             if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
+        if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
             ctx->stack_host = nullptr; ctx->stack_host_bytes = 0;
             const size_t want = 2 * (hdr_off + sizeof(StackHeader));
             FQ_CUDA_OK(cudaMallocHost(&ctx->stack_host, want));
@@ -415,8 +417,28 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
 
 int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)
 {
-    (void)ctx; (void)layer; (void)X_dev; (void)M; (void)ldx; (void)Y_dev; (void)ldy; (void)stream;
-    return FQ_ERR_ARG;
+    if (!ctx || !X_dev || !Y_dev) return FQ_ERR_ARG;
+    if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    const Layer& L = ctx->layers[layer];
+    if (!L.registered || L.active_bits == 0) return FQ_ERR_NOT_PACKED;
+    if (M < 1 || M > (1 << 20) || ldx < L.k_in || ldy < L.n_out || ldx % 8 != 0 || ldy % 8 != 0) return FQ_ERR_SHAPE;
+    if (!aligned(X_dev, 16) || !aligned(Y_dev, 16)) return FQ_ERR_ALIGN;
+    const int bits = L.active_bits;
+    const Variant* v = active_variant(L, bits);
+    if (!v) return FQ_ERR_NO_VARIANT;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    const size_t need = (size_t)L.n_out * L.k_in * 2;
+    if (need > ctx->gemm_ws_bytes) {
+        FQ_CUDA_OK(cudaDeviceSynchronize());
+        if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
+        ctx->gemm_ws = nullptr; ctx->gemm_ws_bytes = 0;
+        FQ_CUDA_OK(cudaMalloc(&ctx->gemm_ws, need));
+        ctx->gemm_ws_bytes = need;
+    }
+    const int zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
+    return launch_gemm(ctx, v->store, blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits), active_fields(L, bits), zero_adjust,
+                       L.n_out, L.k_in, X_dev, M, ldx, Y_dev, ldy, ctx->gemm_ws, (cudaStream_t)stream);
 }
 
 int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* stream)

@@ -68,6 +68,9 @@ struct Ctx {
     size_t stack_dev_bytes = 0;
     char* stack_host = nullptr;  // pinned
     size_t stack_host_bytes = 0;
+    // prefill: dequantised bf16 copy of the layer being multiplied
+    char* gemm_ws = nullptr;
+    size_t gemm_ws_bytes = 0;
     uint64_t config_epoch = 0;
     uint64_t stack_key = 0;      // hash of the op list that is currently uploaded
     bool stack_valid = false;
@@ -97,6 +100,9 @@ int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
 // Units of an op (n_units units, block rotation rot) that CTA `cta` of `grid` processes: [lo, hi).
 void gemv_cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi);
+
+int launch_gemm(Ctx* ctx, const void* store, int blob_stride, const FieldList& fl, int zero_adjust, int n_out, int k_in,
+                const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, void* w_scratch, cudaStream_t st);
 
 }  // namespace fq
 
