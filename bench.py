@@ -124,6 +124,51 @@ def build_stack(P, shapes, bits, device):
     return fq
 
 
+PREFILL_CONFIG_ID = 3
+PREFILL_BITS = [2, 3, 4, 6, 8]
+PREFILL_TOKENS = 4 * 2048
+
+
+def prefill_pass(P, device, blocks, steps, warmup, tokens=PREFILL_TOKENS):
+    """Prefill / calibration-evaluation workload: bf16 activations of 4 x 2048 tokens through every matrix
+    of the 7B-shaped stack (bits seeded from {2,3,4,6,8}), one fq_gemm call per matrix.  Returns a dict."""
+    shapes = S.stack_shapes("7b", blocks)
+    L = len(shapes)
+    bits = S.draw_bits(S.tensor_key(PREFILL_CONFIG_ID, 0, S.TENSOR_BITS), L, PREFILL_BITS)
+    fq = P.FlexQ(L, device.index or 0)
+    for i, (sh, b) in enumerate(zip(shapes, bits)):
+        w = S.weight_rows(S.tensor_key(PREFILL_CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device)
+        c, sc, z = P.fq_quantize_layer(w, int(b))
+        fq.fq_pack_layer(i, c, sc, z, int(b), P.FQ_FMT_PACKED)
+        del w, c, sc, z
+    m = tokens
+    xs = {k: S.activations(S.tensor_key(PREFILL_CONFIG_ID, k, S.TENSOR_X), m, k, torch.bfloat16, device=device)
+          for k in sorted({sh.k_in for sh in shapes})}
+    ys = {n: torch.empty((m, n), dtype=torch.bfloat16, device=device) for n in sorted({sh.n_out for sh in shapes})}
+
+    def one_pass():
+        for i, sh in enumerate(shapes):
+            fq.fq_gemm(i, xs[sh.k_in], ys[sh.n_out])
+
+    for _ in range(warmup):
+        one_pass()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_pass()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    status = fq.fq_status()
+    fq.fq_destroy()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the prefill pass")
+    flop = sum(2.0 * m * sh.n_out * sh.k_in for sh in shapes)
+    return {"ms_per_pass": ms, "tflops": flop / (ms * 1e-3) / 1e12, "flop_per_pass": flop, "tokens": m,
+            "matrices": L, "average_bits": S.average_bits(bits, shapes), "gpu_launches_per_pass": 2 * L}
+
+
 def oracle_sample(shapes, bits, n_layers, device_for_gen):
     """Times the CPU oracle's GEMV on the first `n_layers` matrices of the workload.
     Returns (bytes processed, seconds, description)."""
@@ -179,6 +224,10 @@ def main():
     ap.add_argument("--blocks", type=int, default=32, help="decoder blocks of the 7B-shaped stack (32 = full)")
     ap.add_argument("--ref-layers", type=int, default=7, help="matrices the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the prefill (tensor-core GEMM) leg")
+    ap.add_argument("--prefill-steps", type=int, default=3)
+    ap.add_argument("--prefill-tokens", type=int, default=PREFILL_TOKENS)
+    ap.add_argument("--prefill-only", action="store_true", help="run only the prefill leg and print its object")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -198,6 +247,11 @@ def main():
 
     import paper_2501_07139_b200 as P
     P.lib()                                      # fails loudly if the CUDA library is missing
+
+    if args.prefill_only:
+        pf = prefill_pass(P, device, args.blocks, args.prefill_steps, 3, args.prefill_tokens)
+        print(json.dumps({"prefill_only": pf}), flush=True)
+        return
 
     shapes = S.stack_shapes("7b", args.blocks)
     L = len(shapes)
@@ -304,12 +358,27 @@ def main():
         },
         "clocks": clocks,
     }
+    fq.fq_destroy()
+    del fq
+    torch.cuda.empty_cache()
+    if not args.no_prefill and world == 1:
+        pf = prefill_pass(P, device, args.blocks, args.prefill_steps, 3, args.prefill_tokens)
+        burst, sustained = peaks.get("bf16_tflops", 1590.0), peaks.get("bf16_tflops_sustained", 1400.0)
+        line["prefill"] = {
+            "metric": "prefill dequant-GEMM TFLOP/s", "value": pf["tflops"], "unit": "TFLOP/s", "ms_per_pass": pf["ms_per_pass"],
+            "workload": f"bf16 activations {pf['tokens']} tokens through {pf['matrices']} matrices of the 7B-shaped stack, "
+                        f"bits seeded from {PREFILL_BITS} (average {pf['average_bits']:.2f}), one fq_gemm per matrix",
+            "dtype": "bf16", "gpu_launches_per_pass": pf["gpu_launches_per_pass"],
+            "roofline": {"bound": "tensor", "achieved": pf["tflops"], "peak": sustained, "unit": "TFLOP/s",
+                         "frac": pf["tflops"] / sustained, "peak_kind": f"of {peak_kind} (sustained bf16, the pass is a long step)",
+                         "frac_of_burst": pf["tflops"] / burst, "traffic": None,
+                         "kernel": "gemm_kernel (tcgen05) + dequant_kernel; flops = 2*M*N*K per matrix"},
+        }
     if not args.no_cpu_baseline:
         n_layers = min(args.ref_layers, L)
         byts, secs, desc = oracle_sample(shapes, bits, n_layers, device)
         line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
     print(json.dumps(line), flush=True)
-    fq.fq_destroy()
     if world > 1:
         dist.destroy_process_group()
 
