@@ -13,6 +13,10 @@ namespace {
 
 constexpr size_t kWsHead = 8 * 4096 + 64;      // phase counters (4096 x u64) + exit counter
 constexpr int kMaxPhases = 4096;
+// Workspace layout: [phase counters | exit counter][split-K arrival counters, always zero between launches][partials].
+// Counters and partials never share bytes: a stale partial sum must not be mistaken for an arrival count.
+constexpr size_t kCounterRegion = 4u << 20;
+constexpr size_t kPartialBase = kWsHead + kCounterRegion;
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -147,7 +151,7 @@ int fq_create(fq_ctx** out, int device, int n_layers)
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaMalloc(&ctx->status_dev, sizeof(int)) != cudaSuccess ||
         cudaMemset(ctx->status_dev, 0, sizeof(int)) != cudaSuccess ||
-        ensure_workspace(ctx, kWsHead + (1 << 20)) != FQ_OK) {
+        ensure_workspace(ctx, kPartialBase + (1 << 20)) != FQ_OK) {
         if (ctx->status_dev) cudaFree(ctx->status_dev);
         delete ctx;
         return FQ_ERR_CUDA;
@@ -291,10 +295,11 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
     const size_t pb = op_partial_bytes(op, batch), cb = op_counter_bytes(op);
-    rc = ensure_workspace(ctx, kWsHead + cb + pb + 256);
+    if (cb > kCounterRegion) return FQ_ERR_SHAPE;
+    rc = ensure_workspace(ctx, kPartialBase + pb + 256);
     if (rc != FQ_OK) return rc;
     op.tile_count = reinterpret_cast<unsigned*>(ctx->ws + kWsHead);
-    op.partial = reinterpret_cast<float*>(ctx->ws + kWsHead + round_up((int64_t)cb, 256));
+    op.partial = reinterpret_cast<float*>(ctx->ws + kPartialBase);
     return launch_gemv_single(ctx, op, (cudaStream_t)stream);
 }
 
@@ -358,7 +363,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         GemvOp* ops = reinterpret_cast<GemvOp*>(ctx->stack_host);
         long long* phase_total = reinterpret_cast<long long*>(ctx->stack_host + (size_t)n_ops * sizeof(GemvOp));
         for (int p = 0; p < (n_phases > 0 ? n_phases : 1); p++) phase_total[p] = 0;
-        size_t ws_need = kWsHead;
+        size_t ws_need = kPartialBase, counter_need = 0;
         long long unit_base = 0;
         std::vector<long long> bases(n_ops);
         for (int i = 0; i < n_ops; i++) {
@@ -369,21 +374,18 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             const long long units = (long long)ops[i].n_rp * ops[i].n_chunks;
             unit_base += units;
             if (phases_host) phase_total[phases_host[i]] += units;
-            ws_need = (size_t)round_up((int64_t)ws_need, 256);
-            ws_need += op_counter_bytes(ops[i]);
-            ws_need = (size_t)round_up((int64_t)ws_need, 256);
-            ws_need += op_partial_bytes(ops[i], batch);
+            counter_need += op_counter_bytes(ops[i]);
+            ws_need += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
+        if (counter_need > kCounterRegion) return FQ_ERR_SHAPE;
         int rc = ensure_workspace(ctx, ws_need + 256);
         if (rc != FQ_OK) return rc;
-        size_t off = kWsHead;
+        size_t coff = kWsHead, poff = kPartialBase;
         for (int i = 0; i < n_ops; i++) {
-            off = (size_t)round_up((int64_t)off, 256);
-            ops[i].tile_count = reinterpret_cast<unsigned*>(ctx->ws + off);
-            off += op_counter_bytes(ops[i]);
-            off = (size_t)round_up((int64_t)off, 256);
-            ops[i].partial = reinterpret_cast<float*>(ctx->ws + off);
-            off += op_partial_bytes(ops[i], batch);
+            ops[i].tile_count = reinterpret_cast<unsigned*>(ctx->ws + coff);
+            coff += op_counter_bytes(ops[i]);
+            ops[i].partial = reinterpret_cast<float*>(ctx->ws + poff);
+            poff += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
         // how many units each CTA of the persistent grid will see (the consumers' loop bound)
         int* cta_units = reinterpret_cast<int*>(phase_total + (n_phases > 0 ? n_phases : 1));

@@ -366,6 +366,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 op_seq++;
                 const int op_slot = op_seq % kOpRing;
                 cur.store(reinterpret_cast<GemvOp*>(opring + op_slot * S::kOpBytes), lane);   // for the consumers
+                __threadfence_block();
+                __syncwarp();          // all 32 lanes' words are in place before lane 0 announces the first unit
                 // a PACKED variant's blobs are contiguous: one copy per unit (lane 0); a nested child reads a
                 // prefix of every blob: one copy per blob (lanes 0 .. nb-1)
                 const bool contiguous = op.blob_read == op.blob_stride;

@@ -254,3 +254,26 @@ def test_gemv_argument_errors(P):
                          torch.zeros((4, 1), dtype=torch.float16, device="cuda"), 4)
     assert e.value.code == -3
     fq.fq_destroy()
+
+
+def test_stack_after_single_calls_with_split_k(P):
+    """Split-K arrival counters and partial sums must never share workspace bytes: a per-layer call
+    followed by a stack call over wide layers (several K chunks) once left rows unwritten."""
+    n, k = 1024, 4096
+    fq = P.FlexQ(2)
+    layers = [make_layer(101, i, n, k, 3) for i in range(2)]
+    for i, l in enumerate(layers):
+        fq.fq_pack_layer(i, *to_dev(*l), 3, P.FQ_FMT_PACKED)
+    xs = [x_fp16(101, i, 1, k).cuda() for i in range(2)]
+    y_single = [torch.empty((1, n), dtype=torch.float16, device="cuda") for _ in range(2)]
+    for rep in range(2):
+        for i in range(2):
+            fq.fq_gemv_batched(i, xs[i], y_single[i])
+        ys = [torch.full((1, n), float("nan"), dtype=torch.float16, device="cuda") for _ in range(2)]
+        fq.fq_gemv_stack([0, 1], xs, ys, None, 1)
+        assert fq.fq_status() == 0
+        for i in range(2):
+            assert torch.equal(ys[i], y_single[i])
+    ref = O.gemv(*layers[1], 3, bits_of(xs[1]))
+    assert O.rel_l2(f64_of(y_single[1]), ref) <= GEMV_TOL
+    fq.fq_destroy()
