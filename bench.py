@@ -112,6 +112,16 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(value: float, device) -> float:
+    """The slowest rank's figure (replicas are timed together: barrier, events, max over ranks)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def build_stack(P, shapes, bits, device):
     """Seeded weights -> GPU quantiser -> packed layers.  Returns the context."""
     fq = P.FlexQ(len(shapes), device.index or 0)
@@ -288,12 +298,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1) / steps
-        if world > 1:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1) / steps, device)
 
     def step_dev():
         fq.fq_gemv_stack_raw(args_dep, 1)

@@ -30,38 +30,79 @@ struct DequantArgs {
     __nv_bfloat16* out;              // [n_out][k_in]
 };
 
+// One warp per (row tile, superstep): 16 rows x 256 columns.  The lanes read the stored words exactly as
+// the decode kernel does (coalesced 16-byte chunks), rebuild the codes four at a time (one byte each) and
+// write 8-byte runs of bf16.
+template <int F>
+__device__ __forceinline__ void gather_field(const uint8_t* tile_base, int lane, int shift, uint32_t (&code)[32])
+{
+    constexpr int P = 8 / F;
+    constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
+#pragma unroll
+    for (int jb = 0; jb < F; jb++) {
+        const uint4 w = __ldg(reinterpret_cast<const uint4*>(tile_base + jb * 512 + lane * 16));
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int t = 0; t < P; t++)
+#pragma unroll
+            for (int r = 0; r < 4; r++) code[(P * jb + t) * 4 + r] |= ((ww[r] >> (t * F)) & kMask) << shift;
+    }
+}
+
 __global__ void __launch_bounds__(256) dequant_kernel(const DequantArgs a)
 {
-    const long long per_row = a.k_in / 8;
-    const long long total = (long long)a.n_out * per_row;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const long long n = i / per_row;
-        const int k0 = (int)(i % per_row) * 8;
-        const int rt = (int)(n / kTileRows), r = (int)(n % kTileRows);
-        const int ss = k0 / kStepCols, kk0 = k0 % kStepCols;
+    const int lane = threadIdx.x & 31;
+    const int g = lane >> 2, c = lane & 3;
+    const int n_rt = row_tiles(a.n_out), n_ss = supersteps(a.k_in);
+    const long long total = (long long)n_rt * n_ss;
+    const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (long long ti = warp0; ti < total; ti += n_warps) {
+        const int rt = (int)(ti / n_ss), ss = (int)(ti % n_ss);
         const int tile = rt % kBlobTiles, ssl = ss % kBlobSteps;
         const uint8_t* blob = a.store + ((long long)(rt / kBlobTiles) * a.n_kb + ss / kBlobSteps) * a.blob_stride;
-        const uint32_t mw = *reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile) + ((kk0 >> 7) & 1) * 64 + r * 4);
-        const float s = __half2float(__ushort_as_half((unsigned short)(mw & 0xffffu)));
-        const float z = (float)((int)(mw >> 16) - a.zero_adjust);
-        unsigned code[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        uint32_t code[32];                               // register (k32 step j, a0..a3): four codes, one per byte
+#pragma unroll
+        for (int i = 0; i < 32; i++) code[i] = 0u;
         int prefix = 0;
         for (int fi = 0; fi < a.fl.n; fi++) {
             const int f = a.fl.width[fi];
-            const uint8_t* tile_base = blob + blob_field_off(prefix, f, ssl, tile);
-#pragma unroll
-            for (int e = 0; e < 8; e++) {
-                const FieldPos p = field_pos(f, r, kk0 + e);
-                const uint32_t wv = *reinterpret_cast<const uint32_t*>(tile_base + p.word_byte);
-                code[e] |= ((wv >> p.bit) & ((1u << f) - 1u)) << a.fl.shift[fi];
+            const uint8_t* tb = blob + blob_field_off(prefix, f, ssl, tile);
+            switch (f) {
+                case 8: gather_field<8>(tb, lane, a.fl.shift[fi], code); break;
+                case 4: gather_field<4>(tb, lane, a.fl.shift[fi], code); break;
+                case 2: gather_field<2>(tb, lane, a.fl.shift[fi], code); break;
+                default: gather_field<1>(tb, lane, a.fl.shift[fi], code); break;
             }
             prefix += f;
         }
-        __align__(16) __nv_bfloat16 o[8];
+        const uint32_t* meta = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile));
+        float sc[2][2], zp[2][2];                        // [group][row g / g+8]
 #pragma unroll
-        for (int e = 0; e < 8; e++) o[e] = __float2bfloat16_rn(((float)code[e] - z) * s);
-        *reinterpret_cast<uint4*>(a.out + n * a.k_in + k0) = *reinterpret_cast<const uint4*>(o);
+        for (int grp = 0; grp < 2; grp++)
+#pragma unroll
+            for (int hr = 0; hr < 2; hr++) {
+                const uint32_t m = __ldg(meta + grp * 16 + g + 8 * hr);
+                sc[grp][hr] = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
+                zp[grp][hr] = (float)((int)(m >> 16) - a.zero_adjust);
+            }
+#pragma unroll
+        for (int j = 0; j < 8; j++)
+#pragma unroll
+            for (int r = 0; r < 4; r++) {
+                const int hr = r & 1, half = r >> 1;
+                const long long n = (long long)rt * kTileRows + g + 8 * hr;
+                const int k = ss * kStepCols + 32 * j + 16 * half + 4 * c;
+                if (n >= a.n_out || k >= a.k_in) continue;
+                const uint32_t q4 = code[j * 4 + r];
+                const float s = sc[j >> 2][hr], z = zp[j >> 2][hr];
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(((float)(q4 & 0xffu) - z) * s, ((float)((q4 >> 8) & 0xffu) - z) * s);
+                const __nv_bfloat162 hi = __floats2bfloat162_rn(((float)((q4 >> 16) & 0xffu) - z) * s, ((float)(q4 >> 24) - z) * s);
+                uint2 o;
+                o.x = *reinterpret_cast<const uint32_t*>(&lo);
+                o.y = *reinterpret_cast<const uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(a.out + n * a.k_in + k) = o;
+            }
     }
 }
 
@@ -348,9 +389,9 @@ int launch_gemm(Ctx* ctx, const void* store, int blob_stride, const FieldList& f
     da.store = static_cast<const uint8_t*>(store); da.fl = fl; da.n_out = n_out; da.k_in = k_in;
     da.n_kb = k_blobs(k_in); da.blob_stride = blob_stride; da.zero_adjust = zero_adjust;
     da.out = static_cast<__nv_bfloat16*>(w_scratch);
-    const long long items = (long long)n_out * (k_in / 8);
-    long long blocks = (items + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    const long long items = (long long)row_tiles(n_out) * supersteps(k_in);     // one warp each
+    long long blocks = (items + 7) / 8;
+    if (blocks > 148 * 8) blocks = 148 * 8;
     dequant_kernel<<<(unsigned)blocks, 256, 0, st>>>(da);
     FQ_CUDA_OK(cudaGetLastError());
 
