@@ -179,6 +179,108 @@ def prefill_pass(P, device, blocks, steps, warmup, tokens=PREFILL_TOKENS):
             "matrices": L, "average_bits": S.average_bits(bits, shapes), "gpu_launches_per_pass": 2 * L}
 
 
+def _time_ms(fn, steps, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def config_report(P, device, steps):
+    """The other workloads of the problem statement, one JSON object each (printed by --all-configs):
+    config 0 (one 4096x4096 4-bit layer, rotated over copies larger than L2), config 2 (7B-shaped nested
+    stack, 12-configuration chain) and config 4 (13B-shaped nested stack, 16 configurations, batch 1 / 8
+    decode and prefill at 2048 tokens)."""
+    peaks, kind = measured_peaks()
+    out = []
+    # ---- config 0
+    n = k = 4096
+    copies = 32                                           # 32 x 8.9 MB = 285 MB > 126 MB L2
+    fq = P.FlexQ(copies, device.index or 0)
+    w = S.weight_rows(S.tensor_key(0, 0, S.TENSOR_W), 0, n, k, device=device)
+    c, sc, z = P.fq_quantize_layer(w, 4)
+    for i in range(copies):
+        fq.fq_pack_layer(i, c, sc, z, 4, P.FQ_FMT_PACKED)
+    x = S.activations(S.tensor_key(0, 0, S.TENSOR_X), 1, k).to(device)
+    ys = [torch.empty(n, dtype=torch.float16, device=device) for _ in range(copies)]
+    fp1 = fq.fq_set_config([4] * copies) // copies
+
+    def per_layer():
+        for i in range(copies):
+            fq.fq_gemv(i, x, ys[i])
+    args = fq.stack_args(list(range(copies)), [x] * copies, ys, None)
+    t_call = _time_ms(per_layer, steps) / copies
+    t_stack = _time_ms(lambda: fq.fq_gemv_stack_raw(args, 1), steps) / copies
+    out.append({"config": 0, "workload": "4096x4096 4-bit g=128 GEMV, rotated over 32 stored copies (cold L2)",
+                "footprint_bytes": fp1, "us_per_layer_separate_calls": t_call * 1e3, "us_per_layer_one_launch": t_stack * 1e3,
+                "GBps_separate_calls": fp1 / t_call / 1e6, "GBps_one_launch": fp1 / t_stack / 1e6,
+                "frac_of_measured_hbm_one_launch": fp1 / t_stack / 1e6 / peaks["hbm_gbs"]})
+    fq.fq_destroy()
+    del fq, ys
+    # ---- configs 2 and 4: nested stacks and their chains
+    for cfg, model, n_cfg, hi, lo, floor in ((2, "7b", 12, 7.0, 3.5, 3), (4, "13b", 16, 6.0, 2.5, 2)):
+        shapes = S.stack_shapes(model)
+        L = len(shapes)
+        fq = P.FlexQ(L, device.index or 0)
+        stores = []
+        for i, sh in enumerate(shapes):
+            w = S.weight_rows(S.tensor_key(cfg, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device)
+            c, sc, z = P.fq_quantize_layer(w, 8)
+            stores.append(fq.fq_pack_layer(i, c, sc, z, 8, P.FQ_FMT_PLANES))
+            del w, c, sc, z
+        chain = S.config_chain(S.tensor_key(cfg, 0, S.TENSOR_CHAIN), shapes, n_cfg, hi, lo, floor)
+        phases = S.stack_phases(shapes)
+        rows = []
+        for batch in ((1,) if cfg == 2 else (1, 8)):
+            xs = [S.activations(S.tensor_key(cfg, i, S.TENSOR_X), batch, sh.k_in).to(device) for i, sh in enumerate(shapes)]
+            ys = [torch.empty((batch, sh.n_out), dtype=torch.float16, device=device) for sh in shapes]
+            args_dep = fq.stack_args(list(range(L)), xs, ys, phases)
+            args_free = fq.stack_args(list(range(L)), xs, ys, None)
+            for ci, bits in enumerate(chain):
+                t0 = time.perf_counter()
+                fp = fq.fq_set_config([int(b) for b in bits])
+                switch_us = (time.perf_counter() - t0) * 1e6
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fq.fq_gemv_stack_raw(args_dep, batch); e1.record(); torch.cuda.synchronize()
+                first_ms = e0.elapsed_time(e1)                     # first pass after the switch (table rebuilt)
+                ms = _time_ms(lambda: fq.fq_gemv_stack_raw(args_dep, batch), steps)
+                ms_free = _time_ms(lambda: fq.fq_gemv_stack_raw(args_free, batch), steps)
+                rows.append({"batch": batch, "config_index": ci, "average_bits": S.average_bits(bits, shapes),
+                             "footprint_bytes": fp, "set_config_host_us": switch_us, "first_pass_ms": first_ms,
+                             "ms_per_pass": ms, "GBps": fp / ms / 1e6, "ms_unordered": ms_free, "GBps_unordered": fp / ms_free / 1e6})
+            del xs, ys
+        entry = {"config": cfg, "workload": f"{model}-shaped stack, nested bit-planes, {n_cfg}-configuration chain",
+                 "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0, "decode": rows}
+        if cfg == 4:
+            bits = chain[-1]
+            fq.fq_set_config([int(b) for b in bits])
+            m = 2048
+            xb = {kk: S.activations(S.tensor_key(cfg, kk, S.TENSOR_X), m, kk, torch.bfloat16, device=device)
+                  for kk in sorted({sh.k_in for sh in shapes})}
+            yb = {nn: torch.empty((m, nn), dtype=torch.bfloat16, device=device) for nn in sorted({sh.n_out for sh in shapes})}
+
+            def pf():
+                for i, sh in enumerate(shapes):
+                    fq.fq_gemm(i, xb[sh.k_in], yb[sh.n_out])
+            ms = _time_ms(pf, max(1, steps // 4), 2)
+            flop = sum(2.0 * m * sh.n_out * sh.k_in for sh in shapes)
+            entry["prefill"] = {"tokens": m, "average_bits": S.average_bits(bits, shapes), "ms_per_pass": ms,
+                                "tflops": flop / ms / 1e9, "frac_of_measured_sustained_bf16": flop / ms / 1e9 / peaks["bf16_tflops_sustained"]}
+        if fq.fq_status() != 0:
+            raise RuntimeError("device status after config report")
+        out.append(entry)
+        fq.fq_destroy()
+        del fq, stores
+        torch.cuda.empty_cache()
+    return out
+
+
 def oracle_sample(shapes, bits, n_layers, device_for_gen):
     """Times the CPU oracle's GEMV on the first `n_layers` matrices of the workload.
     Returns (bytes processed, seconds, description)."""
@@ -238,6 +340,8 @@ def main():
     ap.add_argument("--prefill-steps", type=int, default=3)
     ap.add_argument("--prefill-tokens", type=int, default=PREFILL_TOKENS)
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill leg and print its object")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="instead of the bench line, print one JSON object per other workload (configs 0, 2, 4)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -258,6 +362,10 @@ def main():
     import paper_2501_07139_b200 as P
     P.lib()                                      # fails loudly if the CUDA library is missing
 
+    if args.all_configs:
+        for obj in config_report(P, device, max(3, args.steps // 5)):
+            print(json.dumps(obj), flush=True)
+        return
     if args.prefill_only:
         pf = prefill_pass(P, device, args.blocks, args.prefill_steps, 3, args.prefill_tokens)
         print(json.dumps({"prefill_only": pf}), flush=True)
