@@ -116,8 +116,8 @@ int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void
  * until the process exits.  It calls no cudaMalloc / cudaFree and nothing that allocates.
  *   - batch 1 only; x_dev fp16 [k_in], y_dev fp16 [n_out], 16-byte aligned, caller-owned.
  *   - Returns FQ_ERR_SCRATCH (and launches nothing) when the layer at its active width needs
- *     more scratch than the array holds: 4 bytes per 16-row tile plus 64 bytes per
- *     (16-row tile x K chunk).  Every Llama-2-7B / 13B shaped layer fits.
+ *     more scratch than the array holds: 4 bytes per 32-row pair plus 128 bytes per
+ *     (row pair x K chunk of 512..1536 columns).  Every Llama-2-7B / 13B shaped layer fits.
  *   - The first call on a device looks up the array's device address (once per device, with
  *     that device current); make that first call before starting any stream capture.
  *   - All calls share the one array and it keeps whatever the last call left there; the
