@@ -111,19 +111,20 @@ int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void
  * not acceptable for callers such as a real-time serving loop with a fixed memory budget, code
  * running while another library owns the allocator, or a host thread that must never block on
  * the device-wide synchronisation an allocation implies.  This variant keeps its split-K
- * scratch (per-row-tile arrival counters and fp32 partial sums) in a fixed array that is part
- * of the library image: FQ_STATIC_SCRATCH_BYTES on every GPU that loads the library, held
+ * scratch (the partial sums that the K chunks of a row pair exchange) in a fixed array that is
+ * part of the library image: FQ_STATIC_SCRATCH_BYTES on every GPU that loads the library, held
  * until the process exits.  It calls no cudaMalloc / cudaFree and nothing that allocates.
  *   - batch 1 only; x_dev fp16 [k_in], y_dev fp16 [n_out], 16-byte aligned, caller-owned.
  *   - Returns FQ_ERR_SCRATCH (and launches nothing) when the layer at its active width needs
- *     more scratch than the array holds: 4 bytes per 32-row pair plus 128 bytes per
- *     (row pair x K chunk of 512..1536 columns).  Every Llama-2-7B / 13B shaped layer fits.
+ *     more scratch than the array holds: 256 bytes per (32-row pair x K chunk of 512..1536
+ *     columns).  Every Llama-2-7B / 13B shaped layer fits.
  *   - The first call on a device looks up the array's device address (once per device, with
  *     that device current); make that first call before starting any stream capture.
- *   - All calls share the one array and it keeps whatever the last call left there; the
- *     counters are cleared on `stream` before each launch.  Two calls that overlap on the GPU
- *     (different streams, or different contexts) race on it: serialise them. */
-#define FQ_STATIC_SCRATCH_BYTES (1u << 20)
+ *   - All calls share the one array and it keeps whatever the last call left there.  Nothing
+ *     in it has to be cleared: every partial sum carries the tag of the call that wrote it and
+ *     is ignored under any other tag.  Two calls that overlap on the GPU (different streams,
+ *     or different contexts) race on it: serialise them. */
+#define FQ_STATIC_SCRATCH_BYTES (2u << 20)
 int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
 
 /* Decode at batch 1..8:  Y[b][n] = sum_k X[b][k] * w^[n][k].

@@ -13,10 +13,10 @@ namespace {
 
 constexpr size_t kWsHead = 8 * 4096 + 64;      // phase counters (4096 x u64) + exit counter
 constexpr int kMaxPhases = 4096;
-// Workspace layout: [phase counters | exit counter][split-K arrival counters, always zero between launches][partials].
-// Counters and partials never share bytes: a stale partial sum must not be mistaken for an arrival count.
-constexpr size_t kCounterRegion = 4u << 20;
-constexpr size_t kPartialBase = kWsHead + kCounterRegion;
+// Workspace layout: [phase counters | exit counter][split-K partials].  A partial is a 64-bit word (fp32 sum,
+// launch tag); the workspace starts out zeroed and tag 0 is never used, so a word is valid only when its
+// tag equals the tag of the running launch.
+constexpr size_t kPartialBase = kWsHead + 192;
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -84,9 +84,8 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
 size_t op_partial_bytes(const GemvOp& op, int max_batch)
 {
     if (op.n_chunks <= 1) return 0;
-    return (size_t)op.n_rp * op.n_chunks * gemv_partial_floats_per_unit(max_batch) * sizeof(float);
+    return (size_t)op.n_rp * op.n_chunks * gemv_partial_bytes_per_unit(max_batch);
 }
-size_t op_counter_bytes(const GemvOp& op) { return op.n_chunks <= 1 ? 0 : (size_t)round_up(op.n_rp * 4, 16); }
 
 uint64_t hash_mix(uint64_t h, uint64_t v)
 {
@@ -294,12 +293,10 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
     if (rc != FQ_OK) return rc;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
-    const size_t pb = op_partial_bytes(op, batch), cb = op_counter_bytes(op);
-    if (cb > kCounterRegion) return FQ_ERR_SHAPE;
+    const size_t pb = op_partial_bytes(op, batch);
     rc = ensure_workspace(ctx, kPartialBase + pb + 256);
     if (rc != FQ_OK) return rc;
-    op.tile_count = reinterpret_cast<unsigned*>(ctx->ws + kWsHead);
-    op.partial = reinterpret_cast<float*>(ctx->ws + kPartialBase);
+    op.partial = reinterpret_cast<unsigned long long*>(ctx->ws + kPartialBase);
     return launch_gemv_single(ctx, op, (cudaStream_t)stream);
 }
 
@@ -316,7 +313,7 @@ int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_de
     if (rc != FQ_OK) return rc;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
-    return launch_gemv_static(ctx, op, op_counter_bytes(op), op_partial_bytes(op, 1), (cudaStream_t)stream);
+    return launch_gemv_static(ctx, op, op_partial_bytes(op, 1), (cudaStream_t)stream);
 }
 
 int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t* const* x_dev_host,
@@ -354,7 +351,6 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
     if (!(ctx->stack_valid && ctx->stack_key == key)) {
         if (ctx->stack_host_bytes < hdr_off + sizeof(StackHeader)) {
             if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
-        if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
             ctx->stack_host = nullptr; ctx->stack_host_bytes = 0;
             const size_t want = 2 * (hdr_off + sizeof(StackHeader));
             FQ_CUDA_OK(cudaMallocHost(&ctx->stack_host, want));
@@ -363,7 +359,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         GemvOp* ops = reinterpret_cast<GemvOp*>(ctx->stack_host);
         long long* phase_total = reinterpret_cast<long long*>(ctx->stack_host + (size_t)n_ops * sizeof(GemvOp));
         for (int p = 0; p < (n_phases > 0 ? n_phases : 1); p++) phase_total[p] = 0;
-        size_t ws_need = kPartialBase, counter_need = 0;
+        size_t ws_need = kPartialBase;
         long long unit_base = 0;
         std::vector<long long> bases(n_ops);
         for (int i = 0; i < n_ops; i++) {
@@ -371,20 +367,15 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             if (rc != FQ_OK) return rc;
             ops[i].phase = phases_host ? phases_host[i] : -1;
             bases[i] = unit_base;
-            const long long units = (long long)ops[i].n_rp * ops[i].n_chunks;
-            unit_base += units;
-            if (phases_host) phase_total[phases_host[i]] += units;
-            counter_need += op_counter_bytes(ops[i]);
+            unit_base += (long long)ops[i].n_rp * ops[i].n_chunks;
+            if (phases_host) phase_total[phases_host[i]] += ops[i].n_rp;     // one finished row pair = one count
             ws_need += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
-        if (counter_need > kCounterRegion) return FQ_ERR_SHAPE;
         int rc = ensure_workspace(ctx, ws_need + 256);
         if (rc != FQ_OK) return rc;
-        size_t coff = kWsHead, poff = kPartialBase;
+        size_t poff = kPartialBase;
         for (int i = 0; i < n_ops; i++) {
-            ops[i].tile_count = reinterpret_cast<unsigned*>(ctx->ws + coff);
-            coff += op_counter_bytes(ops[i]);
-            ops[i].partial = reinterpret_cast<float*>(ctx->ws + poff);
+            ops[i].partial = reinterpret_cast<unsigned long long*>(ctx->ws + poff);
             poff += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
         // how many units each CTA of the persistent grid will see (the consumers' loop bound)

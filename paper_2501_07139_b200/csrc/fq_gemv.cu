@@ -32,18 +32,29 @@ namespace fq {
 #define FQ_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return FQ_ERR_CUDA; } while (0)
 
 #ifndef FQ_GEMV_WARPS
-#define FQ_GEMV_WARPS 10
+#define FQ_GEMV_WARPS 16
+#endif
+#ifndef FQ_GEMV_TPW
+#define FQ_GEMV_TPW 1
 #endif
 #ifndef FQ_GEMV_UNIT_BYTES
 #define FQ_GEMV_UNIT_BYTES 17408
 #endif
 constexpr int kConsumerWarps = FQ_GEMV_WARPS;
+constexpr int kTilesPerWarp = FQ_GEMV_TPW;             // 16-row tiles of a unit that one consumer warp computes
+constexpr int kWarpsPerUnit = kUnitRowTiles / kTilesPerWarp;
+constexpr int kUnitsInFlight = kConsumerWarps / kWarpsPerUnit;
+static_assert(kTilesPerWarp == 1 || kTilesPerWarp == 2, "a warp computes one or both row tiles of a unit");
+static_assert(kConsumerWarps % kWarpsPerUnit == 0, "consumer warps come in groups of one unit");
 constexpr int kProducerWarp = kConsumerWarps;          // warp index of the producer
 constexpr int kPrepWarp = kConsumerWarps + 1;          // first warp of the activation pre-processors
 constexpr int kPrepWarps = 4;                          // they share the items of a segment
-constexpr int kGemvThreads = (kConsumerWarps + 1 + kPrepWarps) * 32;
+constexpr int kOutputWarp = kPrepWarp + kPrepWarps;    // the warp that owns every global store of results
+constexpr int kGemvThreads = (kConsumerWarps + 1 + kPrepWarps + 1) * 32;
 constexpr int kUnitBytes = FQ_GEMV_UNIT_BYTES;         // bytes of one unit (whole blobs), at most: 2 x 4-bit or 1 x 8-bit blob
-constexpr int kXSlots = 4;                             // activation chunks kept in shared memory
+constexpr int kXSlots = 3;                             // activation chunks kept in shared memory
+constexpr int kOutSlots = 32;                          // finished units waiting for the output warp
+static_assert(kOutSlots <= 32, "the output warp scans one slot per lane");
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 template <int MAXB> struct GemvCfg;
@@ -51,12 +62,24 @@ template <> struct GemvCfg<1> { static constexpr int kBlobsMax = 3; };  // k blo
 template <> struct GemvCfg<8> { static constexpr int kBlobsMax = 1; };
 
 // What the producer tells the consumers: once per op a copy of the op descriptor in a ring ...
-constexpr int kOpRing = 32;                            // > stages: an op slot outlives its last unit
+constexpr int kOpRing = 16;                            // > stages + 1: an op slot outlives the start of its last unit
 // ... and once per unit (next to the stage that holds the unit's weights)
 struct UnitDesc {
-    int ch, rp, nb, seg, op_slot, pad[3];       // K chunk, row pair, blobs in the unit, activation segment, op ring slot
+    int ch, rp, nb, seg;                        // K chunk, row pair, blobs in the unit, activation segment
+    int op_slot;                                // op ring slot
+    int oseq;                                   // >= 0: this unit finishes its row pair, and is the oseq-th such unit of the CTA
+    int pad[2];
 };
 static_assert(sizeof(UnitDesc) == 32, "descriptor layout");
+
+// What a consumer hands to the output warp together with the unit's 32 x batch row sums.
+struct OutDesc {
+    int rp, ch, n_chunks, n_out, phase, batch;
+    uint16_t* y;
+    const unsigned long long* partial;
+    int pad[2];
+};
+static_assert(sizeof(OutDesc) == 48, "descriptor layout");
 
 template <int MAXB> struct GemvSmem {
     static constexpr int kCMax = GemvCfg<MAXB>::kBlobsMax * kBlobSteps;     // supersteps per chunk, at most
@@ -70,7 +93,10 @@ template <int MAXB> struct GemvSmem {
     static constexpr int kXSlotBytes = (kXscaleOff + MAXB * kCMax * 2 * 4 + 127) / 128 * 128;
     static constexpr int kZeroBytes = kCMax * 256 + 64;
     static constexpr int kOpBytes = (int)((sizeof(GemvOp) + 15) / 16 * 16);
-    static constexpr int kFixed = kXSlots * kXSlotBytes + kZeroBytes + kOpRing * kOpBytes + (2 + 2 * kPrepWarps) * kOpBytes + 256;
+    static constexpr int kOutFloats = 32 * (MAXB == 1 ? 1 : 8);              // row sums of one unit
+    static constexpr int kOutBytes = kOutSlots * (kOutFloats * 4 + (int)sizeof(OutDesc));
+    static constexpr int kFixed = kXSlots * kXSlotBytes + kZeroBytes + kOpRing * kOpBytes + (2 + 2 * kPrepWarps) * kOpBytes +
+                                  kOutBytes + 512;
     static constexpr int kPerStage = kStageBytes + (int)sizeof(UnitDesc) + 16 + 4;
     static constexpr int kAuto = (232448 - kFixed) / kPerStage;
     static constexpr int kStages = kAuto > 16 ? 16 : kAuto;
@@ -80,11 +106,15 @@ template <int MAXB> struct GemvSmem {
     static constexpr int oZero = oX + kXSlots * kXSlotBytes;
     static constexpr int oOpRing = oZero + kZeroBytes;               // GemvOp[kOpRing]
     static constexpr int oOpBuf = oOpRing + kOpRing * kOpBytes;   // GemvOp[2] producer, GemvOp[2] per x-prep warp
-    static constexpr int oBars = oOpBuf + (2 + 2 * kPrepWarps) * kOpBytes;   // full[S], empty[S]
-    static constexpr int oReleased = oBars + 2 * kStages * 8;        // u32[S]: uses of a stage that were released
-    static constexpr int oCtl = oReleased + kStages * 4;             // x_ready[XS], x_pending[XS], flags[2]
-    static constexpr int kTotal = oCtl + 64;
+    static constexpr int oOutData = oOpBuf + (2 + 2 * kPrepWarps) * kOpBytes;   // float[kOutSlots][kOutFloats]
+    static constexpr int oOutDesc = oOutData + kOutSlots * kOutFloats * 4;     // OutDesc[kOutSlots]
+    static constexpr int oBars = oOutDesc + kOutSlots * (int)sizeof(OutDesc);  // full[S], empty[S]
+    static constexpr int oReleased = oBars + 2 * kStages * 8;        // u32[S]: consumer warps that released a stage, ever
+    static constexpr int oCtl = oReleased + kStages * 4;             // x_ready[XS], x_pending[XS], flags[2], prep_cmd, pad
+    static constexpr int oOutCtl = oCtl + 64;                        // out_fill[kOutSlots], out_gen[kOutSlots]
+    static constexpr int kTotal = oOutCtl + 2 * kOutSlots * 4 + 16;  // + out_total
     static_assert(kStages >= 4, "decode kernel: no room for a ring");
+    static_assert(kOpRing >= kStages + 2, "an op's ring slot must outlive the units that refer to it");
     static_assert(kTotal <= 232448, "decode kernel: shared memory over the 227 KB per-CTA limit");
 };
 
@@ -99,7 +129,8 @@ int gemv_chunk_blobs(int bits, int batch)
 }
 static_assert(kUnitBytes >= kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * 8, "a unit must hold an 8-bit blob");
 
-size_t gemv_partial_floats_per_unit(int batch) { return batch <= 1 ? 32 : 256; }
+// A split-K partial is one 64-bit word per (row, batch entry): fp32 sum in the low half, launch tag in the high half.
+size_t gemv_partial_bytes_per_unit(int batch) { return (batch <= 1 ? 32 : 256) * sizeof(unsigned long long); }
 
 // ------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -162,18 +193,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// Counter updates that carry their own ordering instead of a separate membar: the release half makes
-// this warp's earlier stores (ordered before it by __syncwarp) visible first, the acquire half orders
-// the loads that follow.
-__device__ __forceinline__ unsigned atom_add_acq_rel_u32(unsigned* p, unsigned v)
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v)
 {
-    unsigned old;
-    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-    return old;
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ void red_add_release_u64(unsigned long long* p, unsigned long long v)
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p)
 {
-    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_add_relaxed_u64(unsigned long long* p, unsigned long long v)
+{
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p)
 {
@@ -211,6 +243,7 @@ struct StackArgs {
     const int* cta_units;                  // units of every CTA (nullptr: single op, computed on the device)
     int* status;
     int n_ops, n_phases;
+    unsigned epoch;                        // tag of this launch's split-K partials (never 0)
 };
 
 // Warp-cooperative fetch of op descriptors with one op of look-ahead: the words of op i+1 travel
@@ -236,7 +269,7 @@ struct OpFetch {
 static_assert(sizeof(GemvOp) <= 256, "op descriptor too large for the two-word fetch");
 
 // ------------------------------------------------------------------------------- one field, one superstep
-// Consumes field width F of up to two row tiles for one superstep: eight k32 steps, the first four
+// Consumes field width F of TILES row tiles for one superstep: eight k32 steps, the first four
 // belong to the first group of 128 columns, the last four to the second.  Adds, per tile / pass / row /
 // group, the integer  2^shift * sum_k field_k * x_int_k  into v.
 //   MAXB == 1 : B columns (2t, 2t+1) carry the digits for bit-offset class t, lane (g, c) ends up with
@@ -244,53 +277,54 @@ static_assert(sizeof(GemvOp) <= 256, "op descriptor too large for the two-word f
 //               data for class t (or at zeros).
 //   MAXB  > 1 : every register is shifted down to class 0; B columns (2b, 2b+1) carry batch entry
 //               4*pass + b; xp[pass] points at this lane's B data.
-template <int F, int MAXB>
-__device__ __forceinline__ void field_step(const uint8_t* f0, const uint8_t* f1, bool two_tiles, bool two_pass,
-                                           int lane, const uint8_t* const (&xp)[4], int xoff, int shift,
-                                           int (&v)[2][2][2][2])
+// With one tile per warp the k32 steps of a group alternate between two accumulators, so that two
+// independent mma chains are in flight.
+template <int F, int MAXB, int TILES>
+__device__ __forceinline__ void field_step(const uint8_t* f0, bool two_pass, int lane, const uint8_t* const (&xp)[4],
+                                           int xoff, int shift, int (&v)[TILES][2][2][2])
 {
     constexpr int P = 8 / F;                                   // A registers stacked in one word
     constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
     constexpr int NP = MAXB == 1 ? 1 : 2;
-    int acc[2][NP][2][4];
+    constexpr int NA = (TILES == 1 && MAXB == 1) ? 2 : 1;      // accumulators per (tile, pass, group)
+    int acc[TILES][NP][2][NA][4];
 #pragma unroll
-    for (int i = 0; i < 2 * NP * 2 * 4; i++) (&acc[0][0][0][0])[i] = 0;
+    for (int i = 0; i < TILES * NP * 2 * NA * 4; i++) (&acc[0][0][0][0][0])[i] = 0;
 
 #pragma unroll
     for (int jb = 0; jb < F; jb++) {
-        const uint4 w0 = *reinterpret_cast<const uint4*>(f0 + jb * 512 + lane * 16);
-        uint4 w1 = make_uint4(0u, 0u, 0u, 0u);
-        if (two_tiles) w1 = *reinterpret_cast<const uint4*>(f1 + jb * 512 + lane * 16);
-        uint4 h0 = w0, h1 = w1;                                // F == 1: classes 4..7 come down by one shift
-        if (F == 1 && MAXB == 1) {
-            h0 = make_uint4(w0.x >> 4, w0.y >> 4, w0.z >> 4, w0.w >> 4);
-            h1 = make_uint4(w1.x >> 4, w1.y >> 4, w1.z >> 4, w1.w >> 4);
+        uint4 w[TILES], h[TILES];
+#pragma unroll
+        for (int tl = 0; tl < TILES; tl++) {
+            w[tl] = *reinterpret_cast<const uint4*>(f0 + tl * F * 512 + jb * 512 + lane * 16);
+            h[tl] = w[tl];                                     // F == 1: classes 4..7 come down by one shift
+            if (F == 1 && MAXB == 1) h[tl] = make_uint4(w[tl].x >> 4, w[tl].y >> 4, w[tl].z >> 4, w[tl].w >> 4);
         }
 #pragma unroll
         for (int t = 0; t < P; t++) {
             const int j = P * jb + t;                          // k32 step inside the superstep
             const int grp = j >> 2;
+            const int ai = NA == 2 ? (j & 1) : 0;
             if (MAXB == 1) {
                 const int tc = (F == 1) ? (t & 3) : t;         // bit-offset class = B column pair
                 const uint32_t m = kMask << (tc * F);
-                const uint4& a = (F == 1 && t >= 4) ? h0 : w0;
-                const uint4& b = (F == 1 && t >= 4) ? h1 : w1;
                 const uint2 x = *reinterpret_cast<const uint2*>(xp[tc] + xoff + j * 32);
-                mma_u8s8(acc[0][0][grp], a.x & m, a.y & m, a.z & m, a.w & m, x.x, x.y);
-                mma_u8s8(acc[1][0][grp], b.x & m, b.y & m, b.z & m, b.w & m, x.x, x.y);
+#pragma unroll
+                for (int tl = 0; tl < TILES; tl++) {
+                    const uint4& a = (F == 1 && t >= 4) ? h[tl] : w[tl];
+                    mma_u8s8(acc[tl][0][grp][ai], a.x & m, a.y & m, a.z & m, a.w & m, x.x, x.y);
+                }
             } else {
                 const int sh = t * F;
-                const uint32_t a0 = (w0.x >> sh) & kMask, a1 = (w0.y >> sh) & kMask;
-                const uint32_t a2 = (w0.z >> sh) & kMask, a3 = (w0.w >> sh) & kMask;
-                const uint32_t b0 = (w1.x >> sh) & kMask, b1 = (w1.y >> sh) & kMask;
-                const uint32_t b2 = (w1.z >> sh) & kMask, b3 = (w1.w >> sh) & kMask;
                 const uint2 x = *reinterpret_cast<const uint2*>(xp[0] + xoff + j * 32);
-                mma_u8s8(acc[0][0][grp], a0, a1, a2, a3, x.x, x.y);
-                mma_u8s8(acc[1][0][grp], b0, b1, b2, b3, x.x, x.y);
-                if (two_pass) {
-                    const uint2 x2 = *reinterpret_cast<const uint2*>(xp[1] + xoff + j * 32);
-                    mma_u8s8(acc[0][NP - 1][grp], a0, a1, a2, a3, x2.x, x2.y);
-                    mma_u8s8(acc[1][NP - 1][grp], b0, b1, b2, b3, x2.x, x2.y);
+                uint2 x2 = make_uint2(0u, 0u);
+                if (two_pass) x2 = *reinterpret_cast<const uint2*>(xp[1] + xoff + j * 32);
+#pragma unroll
+                for (int tl = 0; tl < TILES; tl++) {
+                    const uint32_t a0 = (w[tl].x >> sh) & kMask, a1 = (w[tl].y >> sh) & kMask;
+                    const uint32_t a2 = (w[tl].z >> sh) & kMask, a3 = (w[tl].w >> sh) & kMask;
+                    mma_u8s8(acc[tl][0][grp][0], a0, a1, a2, a3, x.x, x.y);
+                    if (two_pass) mma_u8s8(acc[tl][NP - 1][grp][0], a0, a1, a2, a3, x2.x, x2.y);
                 }
             }
         }
@@ -299,14 +333,16 @@ __device__ __forceinline__ void field_step(const uint8_t* f0, const uint8_t* f1,
     // apply the field's position inside the code
     const int down = MAXB == 1 ? (lane & 3) * F : 0;
 #pragma unroll
-    for (int tile = 0; tile < 2; tile++)
+    for (int tl = 0; tl < TILES; tl++)
 #pragma unroll
         for (int p = 0; p < NP; p++)
 #pragma unroll
             for (int grp = 0; grp < 2; grp++) {
-                const int* a = acc[tile][p][grp];
-                v[tile][p][0][grp] += ((a[0] + (a[1] << 8)) >> down) << shift;
-                v[tile][p][1][grp] += ((a[2] + (a[3] << 8)) >> down) << shift;
+                int a[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) a[i] = acc[tl][p][grp][0][i] + (NA == 2 ? acc[tl][p][grp][NA - 1][i] : 0);
+                v[tl][p][0][grp] += ((a[0] + (a[1] << 8)) >> down) << shift;
+                v[tl][p][1][grp] += ((a[2] + (a[3] << 8)) >> down) << shift;
             }
 }
 
@@ -324,14 +360,19 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
     volatile int* x_pending = x_ready + kXSlots;                               // units that still need the slot
     volatile int* flags = x_pending + kXSlots;                                 // [0]: stop computing, [1]: stop everything
     volatile int* prep_cmd = flags + 2;                                        // decision shared by the pre-processing warps
+    volatile unsigned* out_fill = reinterpret_cast<volatile unsigned*>(smem + S::oOutCtl);   // consumer warps that filled a slot
+    volatile unsigned* out_gen = out_fill + kOutSlots;                         // times the output warp drained a slot
+    volatile int* out_total = reinterpret_cast<volatile int*>(out_gen + kOutSlots);   // finishing units of this CTA (-1: not known yet)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::kStages; s++) {
             mbar_init(bars + 8 * s, 1);
-            mbar_init(bars + 8 * (S::kStages + s), 1);
+            mbar_init(bars + 8 * (S::kStages + s), kWarpsPerUnit);
             released[s] = 0u;
         }
         for (int i = 0; i < kXSlots; i++) { x_ready[i] = 0; x_pending[i] = 0; }
+        for (int i = 0; i < kOutSlots; i++) { out_fill[i] = 0u; out_gen[i] = 0u; }
+        out_total[0] = -1;
         flags[0] = 0; flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -355,6 +396,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
         int stage = 0;                               // ring position and how often the ring wrapped (32-bit state only:
         unsigned wraps = 0;                          // this loop is the serial bottleneck of the CTA)
         int seg = -1, op_seq = -1;
+        int oseq = 0;                                // finishing units issued so far
         bool stop = false;
         for (int oi = 0; oi < sa.n_ops && !stop; oi++) {
             const OpFetch cur = fetch;                                // the words of this op, still in registers
@@ -369,52 +411,74 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 __threadfence_block();
                 __syncwarp();          // all 32 lanes' words are in place before lane 0 announces the first unit
                 // a PACKED variant's blobs are contiguous: one copy per unit (lane 0); a nested child reads a
-                // prefix of every blob: one copy per blob (lanes 0 .. nb-1)
+                // prefix of every blob: one copy per blob (lanes 0 .. nb-1).
+                // Everything the unit loop needs sits in registers and is advanced by additions: this loop
+                // is the serial path that feeds the whole CTA.
+                const int n_rp = op.n_rp, n_kb = op.n_kb, chunk_blobs = op.chunk_blobs, n_chunks = op.n_chunks;
+                const uint32_t blob_read = (uint32_t)op.blob_read;
+                const long long blob_stride = op.blob_stride;
+                const uint8_t* store = op.store;
                 const bool contiguous = op.blob_read == op.blob_stride;
-                const int n_units = hi - lo;
-                int ch = lo / op.n_rp, rp = lo % op.n_rp;
-                bool new_chunk = true;
-                int kb0 = 0, nb = 0;
-                for (int iu = 0; iu < n_units; iu++) {
-                    if (new_chunk) {
-                        seg++;
-                        kb0 = ch * op.chunk_blobs;
-                        nb = min(op.chunk_blobs, op.n_kb - kb0);
-                        new_chunk = false;
-                    }
-                    const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
-                    int ok = 1;
-                    if (lane == 0) {
-                        if (flags[1]) ok = 0;
-                        else if (wraps > 0 && !mbar_wait(empty, (wraps - 1u) & 1u)) {
-                            atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT);
-                            flags[0] = 1; flags[1] = 1;
-                            ok = 0;
+                const long long rp_stride = (long long)n_kb * blob_stride;
+                int ch = lo / n_rp, rp = lo - ch * n_rp;
+                int rpm = rp % n_chunks;                             // rp mod n_chunks, kept up by counting
+                int n_left = hi - lo;
+                while (n_left > 0 && !stop) {
+                    // ---- the units of one K chunk
+                    seg++;
+                    const int kb0 = ch * chunk_blobs;
+                    const int nb = min(chunk_blobs, n_kb - kb0);
+                    const uint32_t bytes = (uint32_t)nb * blob_read;
+                    const uint8_t* src = store + ((long long)rp * n_kb + kb0) * blob_stride;
+                    const int in_chunk = min(n_left, n_rp - rp);
+                    for (int i = 0; i < in_chunk; i++) {
+                        const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
+                        int ok = 1;
+                        if (lane == 0) {
+                            if (wraps > 0 && !mbar_try_wait(empty, (wraps - 1u) & 1u)) {
+                                // the ring is full: the usual case when the consumers wait for activations
+                                if (flags[1]) ok = 0;
+                                else if (!mbar_wait(empty, (wraps - 1u) & 1u)) {
+                                    atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT);
+                                    flags[0] = 1; flags[1] = 1;
+                                    ok = 0;
+                                }
+                            }
+                            if (ok) {
+                                // the chunk that adds up a row pair rotates with the row pair, so that this work
+                                // (and the place in the output queue it needs) is spread evenly over the CTAs
+                                int4* d = reinterpret_cast<int4*>(smem + S::oDesc + stage * (int)sizeof(UnitDesc));
+                                d[0] = make_int4(ch, rp, nb, seg);
+                                d[1] = make_int4(op_slot, ch == rpm ? oseq : -1, 0, 0);
+                                mbar_expect_tx(full, bytes);
+                            }
                         }
-                        if (ok) {
-                            UnitDesc* d = reinterpret_cast<UnitDesc*>(smem + S::oDesc) + stage;
-                            d->ch = ch; d->rp = rp; d->nb = nb; d->seg = seg; d->op_slot = op_slot;
-                            mbar_expect_tx(full, (uint32_t)(nb * op.blob_read));
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) { stop = true; break; }
+                        const uint32_t stage_base = smem_u32(smem + S::oStages) + (uint32_t)stage * S::kStageBytes;
+                        if (contiguous) {
+                            if (lane == 0) bulk_g2s(stage_base, src, bytes, full);
+                        } else if (lane < nb) {
+                            bulk_g2s(stage_base + lane * blob_read, src + lane * blob_stride, blob_read, full);
                         }
+                        if (ch == rpm) oseq++;
+                        if (++rpm == n_chunks) rpm = 0;
+                        if (++stage == S::kStages) { stage = 0; wraps++; }
+                        rp++;
+                        src += rp_stride;
                     }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) { stop = true; break; }
-                    const uint32_t stage_base = smem_u32(smem + S::oStages + stage * S::kStageBytes);
-                    const uint8_t* src = op.store + ((long long)rp * op.n_kb + kb0) * op.blob_stride;
-                    if (contiguous) {
-                        if (lane == 0) bulk_g2s(stage_base, src, nb * op.blob_read, full);
-                    } else if (lane < nb) {
-                        bulk_g2s(stage_base + lane * op.blob_read, src + (long long)lane * op.blob_stride, op.blob_read, full);
-                    }
-                    if (++stage == S::kStages) { stage = 0; wraps++; }
-                    if (++rp == op.n_rp) { rp = 0; ch++; new_chunk = true; }
+                    n_left -= in_chunk;
+                    rp = 0; rpm = 0; ch++;
                 }
+                if (lane == 0 && flags[1]) stop = true;
+                stop = __shfl_sync(0xffffffffu, stop ? 1 : 0, 0) != 0;
             }
             __syncwarp();
             fetch.store(&opbuf[(oi + 1) & 1], lane);
             __syncwarp();
         }
-    } else if (warp >= kPrepWarp) {
+        if (lane == 0 && !stop) out_total[0] = oseq;                // the output warp may leave after this many
+    } else if (warp >= kPrepWarp && warp < kPrepWarp + kPrepWarps) {
         // ================================================================== activation pre-processing
         // All pre-processing warps walk the same list of (op, K chunk) segments and split the
         // (batch row, superstep) items of each segment among them; named barrier 1 keeps them in step.
@@ -544,15 +608,113 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 __threadfence_block();
                 asm volatile("bar.sync 1, %0;" ::"n"(kPrepWarps * 32) : "memory");
                 if (pw == 0 && lane == 0) {
-                    x_pending[slot] = units;
+                    x_pending[slot] = units * kWarpsPerUnit;
                     __threadfence_block();
                     x_ready[slot] = seg + 1;
                 }
             }
         }
+    } else if (warp == kOutputWarp) {
+        // ================================================================== output warp
+        // Finishes row pairs.  The unit whose K chunk is (row pair mod chunks) adds up its row pair: its own
+        // sums arrive through the queue in shared memory, the other chunks' sums are tagged 64-bit words in
+        // global memory (value, launch tag) that their consumers stored without any fence -- a word counts
+        // once its tag is this launch's.  The sums are added in chunk order, so results do not depend on
+        // timing.  One fence per batch of finished row pairs orders y before the phase counter.
+        constexpr int BW = MAXB == 1 ? 1 : 8;                            // result floats per row
+        const float* odata = reinterpret_cast<const float*>(smem + S::oOutData);
+        const OutDesc* odesc = reinterpret_cast<const OutDesc*>(smem + S::oOutDesc);
+        int processed = 0;
+        unsigned long long last_progress = 0ull;
+        unsigned idle_it = 0u;
+        for (;;) {
+            // every decision that ends the loop is taken by lane 0 and broadcast: the lanes must leave together
+            const bool filled = lane < kOutSlots && out_fill[lane] == (unsigned)kWarpsPerUnit;
+            const unsigned m = __ballot_sync(0xffffffffu, filled);
+            unsigned done = 0u;
+            if (m) {
+                __threadfence_block();                                   // the slots' contents after their fill counts
+                for (unsigned mm = m; mm; mm &= mm - 1u) {
+                    const int s = __ffs(mm) - 1;
+                    const OutDesc& d = odesc[s];
+                    const float* o = odata + s * S::kOutFloats;
+                    float sum[BW];
+                    bool ok = true;
+#pragma unroll
+                    for (int i = 0; i < BW; i++) {
+                        const int e = lane + 32 * i;                     // e = local row * BW + batch entry
+                        const unsigned long long* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW) + e;
+                        float acc = 0.f;
+                        for (int q0 = 0; q0 < d.n_chunks; q0 += 8) {
+                            unsigned long long w[8];
+#pragma unroll
+                            for (int j = 0; j < 8; j++) {
+                                const int q = q0 + j;
+                                w[j] = 0ull;
+                                if (q < d.n_chunks && q != d.ch) w[j] = ld_relaxed_u64(pt + (long long)q * (32 * BW));
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; j++) {
+                                const int q = q0 + j;
+                                if (q >= d.n_chunks) break;
+                                if (q == d.ch) acc += o[e];
+                                else {
+                                    ok = ok && (unsigned)(w[j] >> 32) == sa.epoch;
+                                    acc += __uint_as_float((unsigned)w[j]);
+                                }
+                            }
+                        }
+                        sum[i] = acc;
+                    }
+                    if (!__all_sync(0xffffffffu, ok)) continue;          // some chunk has not arrived yet: look again later
+                    const int row_base = d.rp * (kUnitRowTiles * kTileRows);
+                    __half* y = reinterpret_cast<__half*>(d.y);
+#pragma unroll
+                    for (int i = 0; i < BW; i++) {
+                        const int e = lane + 32 * i;
+                        const int row = row_base + e / BW, b = e % BW;
+                        if (row < d.n_out && b < d.batch) y[(long long)b * d.n_out + row] = __float2half_rn(sum[i]);
+                    }
+                    done |= 1u << s;
+                }
+            }
+            if (done) {
+                __syncwarp();
+                __threadfence();                                         // y before the phase counter
+                if ((done >> lane) & 1u) {
+                    const int phase = odesc[lane].phase;
+                    if (phase >= 0) red_add_relaxed_u64(sa.phase_done + phase, 1ull);
+                    out_fill[lane] = 0u;                                 // hand the slot back
+                    __threadfence_block();
+                    out_gen[lane] = out_gen[lane] + 1u;
+                }
+                processed += __popc(done);
+                last_progress = 0ull; idle_it = 0u;
+                continue;
+            }
+            int leave = 0;
+            if (lane == 0) {
+                const int want = out_total[0];
+                if (flags[0] || (want >= 0 && processed >= want)) leave = 1;
+                else if ((++idle_it & 127u) == 0u) {
+                    const unsigned long long now = global_ns();
+                    if (last_progress == 0ull) last_progress = now;
+                    else if (now - last_progress > kWaitLimitNs) {
+                        atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1;
+                        leave = 1;
+                    }
+                }
+            }
+            if (__shfl_sync(0xffffffffu, leave, 0)) break;
+            __nanosleep(m ? 100 : 32);
+        }
     } else {
         // ================================================================== consumers
+        // kWarpsPerUnit warps share a unit, each computes kTilesPerWarp of its two 16-row tiles.
         const int g = lane >> 2, c = lane & 3;
+        const int uidx = warp / kWarpsPerUnit;                       // which of the units in flight
+        const int tile0 = (warp % kWarpsPerUnit) * kTilesPerWarp;    // first row tile of this warp
+        constexpr int TL = kTilesPerWarp;
         const uint8_t* zero_page = smem + S::oZero + c * 8;
         int total = 0;                               // units of this CTA over the whole launch
         if (sa.cta_units) total = sa.cta_units[cta];
@@ -562,187 +724,198 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
             total = hi - lo;
         }
         const uint8_t* opring = smem + S::oOpRing;
+        float* odata = reinterpret_cast<float*>(smem + S::oOutData);
+        OutDesc* odesc = reinterpret_cast<OutDesc*>(smem + S::oOutDesc);
         bool stop = false;
-        {
-            for (int seq = warp; seq < total && !stop; seq += kConsumerWarps) {
-                if (flags[1]) { stop = true; break; }
-                const int stage = seq % S::kStages;
-                const unsigned use = (unsigned)(seq / S::kStages);
-                const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
-                // a stage's uses are consumed strictly in order: wait for the release of the previous
-                // use before trusting the parity of the full barrier
-                bool ok = true;
-                if (use > 0) ok = smem_wait([&] { return released[stage] >= use || flags[1]; });
-                if (ok && !flags[1]) ok = mbar_wait(full, use & 1u);
-                if (!ok || flags[1]) {
-                    if (lane == 0 && !ok) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1; }
+        for (int seq = uidx; seq < total && !stop; seq += kUnitsInFlight) {
+            if (flags[1]) { stop = true; break; }
+            const int stage = seq % S::kStages;
+            const unsigned use = (unsigned)(seq / S::kStages);
+            const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
+            // a stage's uses are consumed strictly in order: wait for the release of the previous
+            // use before trusting the parity of the full barrier
+            bool ok = true;
+            if (use > 0) ok = smem_wait([&] { return released[stage] >= use * kWarpsPerUnit || flags[1]; });
+            if (ok && !flags[1]) ok = mbar_wait(full, use & 1u);
+            if (!ok || flags[1]) {
+                if (lane == 0 && !ok) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1; }
+                stop = true;
+                break;
+            }
+            // (field widths and shifts travel as packed nibbles: a byte array indexed in the loop below
+            // would live in local memory)
+            struct { int ch, rp, cnt, seg, blob_read, n_fields, zero_adjust, batch, op_slot, oseq, n_chunks;
+                     unsigned long long* partial; uint32_t widths, shifts; } d;
+            {
+                const UnitDesc ud = *(reinterpret_cast<const UnitDesc*>(smem + S::oDesc) + stage);
+                const GemvOp& od = *reinterpret_cast<const GemvOp*>(opring + ud.op_slot * S::kOpBytes);
+                d.ch = ud.ch; d.rp = ud.rp; d.cnt = ud.nb * kBlobSteps; d.seg = ud.seg; d.op_slot = ud.op_slot;
+                d.blob_read = od.blob_read; d.n_fields = od.n_fields;
+                d.zero_adjust = od.zero_adjust; d.batch = od.batch;
+                d.oseq = ud.oseq; d.n_chunks = od.n_chunks; d.partial = od.partial;
+                d.widths = 0u; d.shifts = 0u;
+#pragma unroll
+                for (int i = 0; i < kMaxFields; i++) {
+                    d.widths |= (uint32_t)od.field_width[i] << (4 * i);
+                    d.shifts |= (uint32_t)od.field_shift[i] << (4 * i);
+                }
+            }
+            // a unit that finishes its row pair needs a place in the output queue: that place must be free
+            // again; the descriptor goes there now, while the op's slot in the op ring is certainly still valid
+            const int oslot = d.oseq % kOutSlots;
+            if (d.oseq >= 0) {
+                const unsigned ogen = (unsigned)(d.oseq / kOutSlots);
+                if (!smem_wait([&] { return out_gen[oslot] == ogen || flags[1]; })) {
+                    if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1; }
                     stop = true;
                     break;
                 }
-                struct { int ch, rp, cnt, seg, n_out, n_chunks, blob_read, n_fields, phase, zero_adjust, batch;
-                         uint16_t* y; float* partial; unsigned* tile_count; uint8_t width[8], shift[8]; } d;
-                {
-                    const UnitDesc ud = *(reinterpret_cast<const UnitDesc*>(smem + S::oDesc) + stage);
-                    const GemvOp& od = *reinterpret_cast<const GemvOp*>(opring + ud.op_slot * S::kOpBytes);
-                    d.ch = ud.ch; d.rp = ud.rp; d.cnt = ud.nb * kBlobSteps; d.seg = ud.seg;
-                    d.n_out = od.n_out; d.n_chunks = od.n_chunks; d.blob_read = od.blob_read; d.n_fields = od.n_fields;
-                    d.phase = od.phase; d.zero_adjust = od.zero_adjust; d.batch = od.batch;
-                    d.y = od.y; d.partial = od.partial; d.tile_count = od.tile_count;
+                if (flags[1]) { stop = true; break; }
+                if (tile0 == 0 && lane == 0) {
+                    const GemvOp& od = *reinterpret_cast<const GemvOp*>(opring + d.op_slot * S::kOpBytes);
+                    OutDesc& q = odesc[oslot];
+                    q.rp = d.rp; q.ch = d.ch; q.n_chunks = od.n_chunks; q.n_out = od.n_out; q.phase = od.phase; q.batch = od.batch;
+                    q.y = od.y; q.partial = od.partial;
+                }
+            }
+            const uint8_t* st = smem + S::oStages + stage * S::kStageBytes;
+            const int slot = d.seg % kXSlots;
+            if (!smem_wait([&] { return x_ready[slot] == d.seg + 1 || flags[1]; })) {
+                if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; }
+            }
+            __threadfence_block();
+            __syncwarp();
+            const bool live = !flags[0];
+            const int B = d.batch;
+            const bool two_pass = MAXB > 1 && B > 4;
+            const uint8_t* xs = smem + S::oX + slot * S::kXSlotBytes;
+
+            float tot[TL][NP][2];
 #pragma unroll
-                    for (int i = 0; i < kMaxFields; i++) { d.width[i] = od.field_width[i]; d.shift[i] = od.field_shift[i]; }
+            for (int i = 0; i < TL * NP * 2; i++) (&tot[0][0][0])[i] = 0.f;
+
+            if (live) {
+                // this lane's B-operand sources.  B column n = g holds digit (g & 1) of
+                //   batch 1: bit-offset class g >> 1            batch > 1: batch entry 4 * pass + (g >> 1)
+                const uint8_t* xp[4];
+                if (MAXB == 1) {
+#pragma unroll
+                    for (int t = 0; t < 4; t++)
+                        xp[t] = (g >> 1) == t ? xs + (g & 1) * S::kDigitOff + c * 8 : zero_page;
+                } else {
+#pragma unroll
+                    for (int p = 0; p < 2; p++) {
+                        const int b = 4 * p + (g >> 1);
+                        xp[p] = b < B ? xs + b * S::kXRow + (g & 1) * S::kDigitOff + c * 8 : zero_page;
+                    }
+                    xp[2] = zero_page; xp[3] = zero_page;
                 }
-                const uint8_t* st = smem + S::oStages + stage * S::kStageBytes;
-                const int slot = d.seg % kXSlots;
-                if (!smem_wait([&] { return x_ready[slot] == d.seg + 1 || flags[1]; })) {
-                    if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; }
+                const int* xsum = reinterpret_cast<const int*>(xs + S::kXsumOff);
+                const float* xscale = reinterpret_cast<const float*>(xs + S::kXscaleOff);
+                for (int s = 0; s < d.cnt; s++) {
+                    const uint8_t* blob = st + (s / kBlobSteps) * d.blob_read;       // this superstep's blob (prefix)
+                    const int ssl = s % kBlobSteps;
+                    const uint32_t* meta_s = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile0));
+                    int v[TL][2][2][2];
+#pragma unroll
+                    for (int i = 0; i < TL * 8; i++) (&v[0][0][0][0])[i] = 0;
+                    int prefix = 0;
+                    for (int fi = 0; fi < d.n_fields; fi++) {
+                        const int f = (d.widths >> (4 * fi)) & 15, fshift = (d.shifts >> (4 * fi)) & 15;
+                        const uint8_t* f0 = blob + blob_field_off(prefix, f, ssl, tile0);
+                        switch (f) {
+                            case 8: field_step<8, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
+                            case 4: field_step<4, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
+                            case 2: field_step<2, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
+                            default: field_step<1, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
+                        }
+                        prefix += f;
+                    }
+                    // group epilogue: y += s * 2^-e * (v - z * sum x_int)
+#pragma unroll
+                    for (int tl = 0; tl < TL; tl++) {
+#pragma unroll
+                        for (int grp = 0; grp < 2; grp++) {
+                            const uint32_t m0 = meta_s[tl * 32 + grp * 16 + g];
+                            const uint32_t m1 = meta_s[tl * 32 + grp * 16 + g + 8];
+                            const float s0 = __half2float(__ushort_as_half((unsigned short)(m0 & 0xffffu)));
+                            const float s1 = __half2float(__ushort_as_half((unsigned short)(m1 & 0xffffu)));
+                            const int z0 = (int)(m0 >> 16) - d.zero_adjust;
+                            const int z1 = (int)(m1 >> 16) - d.zero_adjust;
+#pragma unroll
+                            for (int p = 0; p < NP; p++) {
+                                // batch 1: only the class-0 lane subtracts the zero-point term
+                                const int b = MAXB == 1 ? 0 : 4 * p + c;
+                                const bool has = MAXB == 1 ? true : b < B;
+                                const int xsm = (MAXB == 1 ? c == 0 : has) ? xsum[b * (S::kCMax * 2) + s * 2 + grp] : 0;
+                                const float sc = has ? xscale[b * (S::kCMax * 2) + s * 2 + grp] : 0.f;
+                                tot[tl][p][0] = fmaf((float)(v[tl][p][0][grp] - z0 * xsm), s0 * sc, tot[tl][p][0]);
+                                tot[tl][p][1] = fmaf((float)(v[tl][p][1][grp] - z1 * xsm), s1 * sc, tot[tl][p][1]);
+                            }
+                        }
+                    }
                 }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                atomicAdd(const_cast<unsigned*>(&released[stage]), 1u);
                 __threadfence_block();
-                __syncwarp();
-                const bool live = !flags[0];
-                const int B = d.batch;
-                const bool two_tiles = true, two_pass = MAXB > 1 && B > 4;
-                const uint8_t* xs = smem + S::oX + slot * S::kXSlotBytes;
+                mbar_arrive(empty);                              // the stage may be refilled
+                atomicSub(const_cast<int*>(&x_pending[slot]), 1);   // one warp fewer needs the activation slot
+            }
+            if (!live) continue;
 
-                float tot[2][NP][2];
+            if (MAXB == 1) {                                     // add up the bit-offset classes held by the quad
 #pragma unroll
-                for (int i = 0; i < 2 * NP * 2; i++) (&tot[0][0][0])[i] = 0.f;
-
-                if (live) {
-                    // this lane's B-operand sources.  B column n = g holds digit (g & 1) of
-                    //   batch 1: bit-offset class g >> 1            batch > 1: batch entry 4 * pass + (g >> 1)
-                    const uint8_t* xp[4];
-                    if (MAXB == 1) {
+                for (int tl = 0; tl < TL; tl++)
 #pragma unroll
-                        for (int t = 0; t < 4; t++)
-                            xp[t] = (g >> 1) == t ? xs + (g & 1) * S::kDigitOff + c * 8 : zero_page;
-                    } else {
-#pragma unroll
-                        for (int p = 0; p < 2; p++) {
-                            const int b = 4 * p + (g >> 1);
-                            xp[p] = b < B ? xs + b * S::kXRow + (g & 1) * S::kDigitOff + c * 8 : zero_page;
-                        }
-                        xp[2] = zero_page; xp[3] = zero_page;
+                    for (int r = 0; r < 2; r++) {
+                        float t = tot[tl][0][r];
+                        t += __shfl_xor_sync(0xffffffffu, t, 1);
+                        t += __shfl_xor_sync(0xffffffffu, t, 2);
+                        tot[tl][0][r] = t;
                     }
-                    const int* xsum = reinterpret_cast<const int*>(xs + S::kXsumOff);
-                    const float* xscale = reinterpret_cast<const float*>(xs + S::kXscaleOff);
-                    for (int s = 0; s < d.cnt; s++) {
-                        const uint8_t* blob = st + (s / kBlobSteps) * d.blob_read;       // this superstep's blob (prefix)
-                        const int ssl = s % kBlobSteps;
-                        const uint32_t* meta_s = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, 0));
-                        int v[2][2][2][2];
-#pragma unroll
-                        for (int i = 0; i < 16; i++) (&v[0][0][0][0])[i] = 0;
-                        int prefix = 0;
-                        for (int fi = 0; fi < d.n_fields; fi++) {
-                            const int f = d.width[fi];
-                            const uint8_t* f0 = blob + blob_field_off(prefix, f, ssl, 0);
-                            const uint8_t* f1 = f0 + f * 512;
-                            switch (f) {
-                                case 8: field_step<8, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
-                                case 4: field_step<4, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
-                                case 2: field_step<2, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
-                                default: field_step<1, MAXB>(f0, f1, two_tiles, two_pass, lane, xp, s * 256, d.shift[fi], v); break;
-                            }
-                            prefix += f;
-                        }
-                        // group epilogue: y += s * 2^-e * (v - z * sum x_int)
-#pragma unroll
-                        for (int tile = 0; tile < 2; tile++) {
-                            if (tile == 1 && !two_tiles) break;
-#pragma unroll
-                            for (int grp = 0; grp < 2; grp++) {
-                                const uint32_t m0 = meta_s[tile * 32 + grp * 16 + g];
-                                const uint32_t m1 = meta_s[tile * 32 + grp * 16 + g + 8];
-                                const float s0 = __half2float(__ushort_as_half((unsigned short)(m0 & 0xffffu)));
-                                const float s1 = __half2float(__ushort_as_half((unsigned short)(m1 & 0xffffu)));
-                                const int z0 = (int)(m0 >> 16) - d.zero_adjust;
-                                const int z1 = (int)(m1 >> 16) - d.zero_adjust;
-#pragma unroll
-                                for (int p = 0; p < NP; p++) {
-                                    // batch 1: only the class-0 lane subtracts the zero-point term
-                                    const int b = MAXB == 1 ? 0 : 4 * p + c;
-                                    const bool has = MAXB == 1 ? true : b < B;
-                                    const int xsm = (MAXB == 1 ? c == 0 : has) ? xsum[b * (S::kCMax * 2) + s * 2 + grp] : 0;
-                                    const float sc = has ? xscale[b * (S::kCMax * 2) + s * 2 + grp] : 0.f;
-                                    tot[tile][p][0] = fmaf((float)(v[tile][p][0][grp] - z0 * xsm), s0 * sc, tot[tile][p][0]);
-                                    tot[tile][p][1] = fmaf((float)(v[tile][p][1][grp] - z1 * xsm), s1 * sc, tot[tile][p][1]);
-                                }
-                            }
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    released[stage] = use + 1u;
-                    __threadfence_block();
-                    mbar_arrive(empty);                              // the stage may be refilled
-                    atomicSub(const_cast<int*>(&x_pending[slot]), 1);   // one unit fewer needs the activation slot
-                }
-                if (!live) continue;
+            }
 
-                if (MAXB == 1) {                                     // add up the bit-offset classes held by the quad
+            // ---- the row sums: value (tile, pass, r) of lane (g, c) belongs to local row tile * 16 + g + 8 r,
+            //      batch entry 0 (batch 1: every lane of the quad holds it) or 4 pass + c
+            constexpr int BW = MAXB == 1 ? 1 : 8;
+            if (d.oseq >= 0) {
+                // this unit finishes its row pair: hand the sums to the output warp
+                float* o = odata + oslot * S::kOutFloats;
 #pragma unroll
-                    for (int tile = 0; tile < 2; tile++)
+                for (int tl = 0; tl < TL; tl++)
+#pragma unroll
+                    for (int p = 0; p < NP; p++)
 #pragma unroll
                         for (int r = 0; r < 2; r++) {
-                            float t = tot[tile][0][r];
-                            t += __shfl_xor_sync(0xffffffffu, t, 1);
-                            t += __shfl_xor_sync(0xffffffffu, t, 2);
-                            tot[tile][0][r] = t;
+                            const int lr = (tile0 + tl) * 16 + g + 8 * r;
+                            if (MAXB == 1) { if (c == 0) o[lr] = tot[tl][0][r]; }
+                            else o[lr * BW + 4 * p + c] = tot[tl][p][r];
                         }
-                }
-
-                // ---- output: direct, or through split-K partials combined by the last arriver
-                // value (tile, pass, r) of lane (g, c): row = (2 rp + tile) * 16 + g + 8 r,
-                //   batch entry = 0 (batch 1, lane c == 0 only) or 4 pass + c
-                __half* y = reinterpret_cast<__half*>(d.y);
-                constexpr int BW = MAXB == 1 ? 1 : 8;                // partial floats per row
-                const int row_base = d.rp * (kUnitRowTiles * kTileRows);
-                bool wrote_final = true;
-                if (d.n_chunks == 1) {
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) atomicAdd(const_cast<unsigned*>(&out_fill[oslot]), 1u);
+            } else {
+                // another unit finishes it: publish tagged words (value, launch tag), fire and forget
+                unsigned long long* pu = d.partial + ((long long)d.rp * d.n_chunks + d.ch) * (32 * BW);
+                const unsigned long long tag = (unsigned long long)sa.epoch << 32;
 #pragma unroll
-                    for (int tile = 0; tile < 2; tile++)
+                for (int tl = 0; tl < TL; tl++) {
+                    if (MAXB == 1) {
+                        if (c < 2) {                                 // lane c of the quad stores row g + 8 c
+                            const float v = c == 0 ? tot[tl][0][0] : tot[tl][0][1];
+                            st_relaxed_u64(pu + (tile0 + tl) * 16 + g + 8 * c, tag | __float_as_uint(v));
+                        }
+                    } else {
 #pragma unroll
                         for (int p = 0; p < NP; p++)
 #pragma unroll
                             for (int r = 0; r < 2; r++) {
-                                const int row = row_base + tile * 16 + g + 8 * r;
-                                const int b = MAXB == 1 ? 0 : 4 * p + c;
-                                const bool mine = MAXB == 1 ? c == 0 : b < B;
-                                if (mine && row < d.n_out) y[(long long)b * d.n_out + row] = __float2half_rn(tot[tile][p][r]);
+                                const int lr = (tile0 + tl) * 16 + g + 8 * r;
+                                st_relaxed_u64(pu + lr * BW + 4 * p + c, tag | __float_as_uint(tot[tl][p][r]));
                             }
-                } else {
-                    float* pu = d.partial + ((long long)d.rp * d.n_chunks + d.ch) * (32 * BW);
-#pragma unroll
-                    for (int tile = 0; tile < 2; tile++)
-#pragma unroll
-                        for (int p = 0; p < NP; p++)
-#pragma unroll
-                            for (int r = 0; r < 2; r++) {
-                                const int lr = tile * 16 + g + 8 * r;
-                                if (MAXB == 1) { if (c == 0) pu[lr] = tot[tile][0][r]; }
-                                else pu[lr * BW + 4 * p + c] = tot[tile][p][r];
-                            }
-                    __syncwarp();
-                    unsigned old = 0;
-                    if (lane == 0) old = atom_add_acq_rel_u32(d.tile_count + d.rp, 1u);
-                    old = __shfl_sync(0xffffffffu, old, 0);
-                    wrote_final = false;
-                    if (old == (unsigned)(d.n_chunks - 1)) {
-                        const float* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW);
-                        for (int e = lane; e < 32 * BW; e += 32) {   // e = local row * BW + batch entry
-                            float sum = 0.f;
-                            for (int q = 0; q < d.n_chunks; q++) sum += __ldcg(pt + (long long)q * (32 * BW) + e);
-                            const int row = row_base + e / BW, b = e % BW;
-                            if (row < d.n_out && b < B) y[(long long)b * d.n_out + row] = __float2half_rn(sum);
-                        }
-                        if (lane == 0) d.tile_count[d.rp] = 0u;      // ready for the next launch
-                        wrote_final = true;
                     }
-                }
-                if (d.phase >= 0) {
-                    __syncwarp();                                    // y is ordered before the release below
-                    if (lane == 0) red_add_release_u64(sa.phase_done + d.phase, 1ull);
                 }
             }
         }
@@ -761,9 +934,10 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
 }
 
 // ------------------------------------------------------------------------------- launchers
+// The launch is always cooperative: a CTA that finishes a row pair waits (bounded) for sums that other
+// CTAs produce, so all CTAs of the grid have to be resident together.
 template <int MAXB>
-static int launch_impl(Ctx* ctx, const GemvOp& single, const StackArgs& sa, long long total_units, bool cooperative,
-                       cudaStream_t st)
+static int launch_impl(Ctx* ctx, const GemvOp& single, const StackArgs& sa, long long total_units, cudaStream_t st)
 {
     using S = GemvSmem<MAXB>;
     static bool configured[64] = {};
@@ -774,15 +948,17 @@ static int launch_impl(Ctx* ctx, const GemvOp& single, const StackArgs& sa, long
     long long blocks = ctx->sm_count;
     if (total_units < blocks) blocks = total_units;
     if (blocks < 1) return FQ_OK;
-    if (cooperative) {
-        void* args[] = {(void*)&single, (void*)&sa};
-        FQ_CUDA_OK(cudaLaunchCooperativeKernel((const void*)gemv_kernel<MAXB>, dim3((unsigned)blocks), dim3(kGemvThreads),
-                                               args, S::kTotal, st));
-    } else {
-        gemv_kernel<MAXB><<<(unsigned)blocks, kGemvThreads, S::kTotal, st>>>(single, sa);
-        FQ_CUDA_OK(cudaGetLastError());
-    }
+    void* args[] = {(void*)&single, (void*)&sa};
+    FQ_CUDA_OK(cudaLaunchCooperativeKernel((const void*)gemv_kernel<MAXB>, dim3((unsigned)blocks), dim3(kGemvThreads),
+                                           args, S::kTotal, st));
     return FQ_OK;
+}
+
+// Tag for the split-K partials of the next launch that uses the context's workspace.
+static unsigned next_epoch(unsigned& e)
+{
+    if (++e == 0u) ++e;                        // 0 marks words that no launch has written
+    return e;
 }
 
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st)
@@ -792,8 +968,9 @@ int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st)
     sa.status = ctx->status_dev;
     sa.n_ops = 1;
     sa.n_phases = 0;
+    sa.epoch = next_epoch(ctx->launch_epoch);
     const long long units = (long long)op.n_rp * op.n_chunks;
-    return op.batch <= 1 ? launch_impl<1>(ctx, op, sa, units, false, st) : launch_impl<8>(ctx, op, sa, units, false, st);
+    return op.batch <= 1 ? launch_impl<1>(ctx, op, sa, units, st) : launch_impl<8>(ctx, op, sa, units, st);
 }
 
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st)
@@ -808,10 +985,10 @@ int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, i
     sa.status = ctx->status_dev;
     sa.n_ops = hdr.n_ops;
     sa.n_phases = hdr.n_phases;
+    sa.epoch = next_epoch(ctx->launch_epoch);
     GemvOp dummy{};
-    const bool coop = hdr.n_phases > 0;
-    return max_batch <= 1 ? launch_impl<1>(ctx, dummy, sa, hdr.total_units, coop, st)
-                          : launch_impl<8>(ctx, dummy, sa, hdr.total_units, coop, st);
+    return max_batch <= 1 ? launch_impl<1>(ctx, dummy, sa, hdr.total_units, st)
+                          : launch_impl<8>(ctx, dummy, sa, hdr.total_units, st);
 }
 
 // ------------------------------------------------------------------------------- allocation-free variant
@@ -833,24 +1010,25 @@ static int static_scratch_address(int device, unsigned char** out)
     return FQ_OK;
 }
 
-// Runs one batch-1 decode op with counters and partials placed in the built-in array.
-int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st)
+// Runs one batch-1 decode op with its split-K partials placed in the built-in array.
+// The array keeps the previous call's contents.  Nothing in it has to start at zero: a partial is
+// only believed when it carries this call's tag, and the tags of the calls that share the array
+// (all contexts on a device) come from one counter per device.
+int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st)
 {
-    const size_t counters = (size_t)round_up((int64_t)counter_bytes, 256);
-    if (counters + partial_bytes > FQ_STATIC_SCRATCH_BYTES) return FQ_ERR_SCRATCH;
+    static unsigned epoch[64] = {};
+    if (partial_bytes > FQ_STATIC_SCRATCH_BYTES) return FQ_ERR_SCRATCH;
     unsigned char* base = nullptr;
     const int rc = static_scratch_address(ctx->device, &base);
     if (rc != FQ_OK) return rc;
-    op.tile_count = reinterpret_cast<unsigned*>(base);
-    op.partial = reinterpret_cast<float*>(base + counters);
-    // the array keeps the previous call's contents: arrival counters must start at zero
-    if (counter_bytes) FQ_CUDA_OK(cudaMemsetAsync(base, 0, counter_bytes, st));
+    op.partial = reinterpret_cast<unsigned long long*>(base);
     StackArgs sa{};
     sa.table = nullptr;
     sa.status = ctx->status_dev;
     sa.n_ops = 1;
     sa.n_phases = 0;
-    return launch_impl<1>(ctx, op, sa, (long long)op.n_rp * op.n_chunks, false, st);
+    sa.epoch = next_epoch(epoch[ctx->device]);
+    return launch_impl<1>(ctx, op, sa, (long long)op.n_rp * op.n_chunks, st);
 }
 
 }  // namespace fq

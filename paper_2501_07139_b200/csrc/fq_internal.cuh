@@ -35,8 +35,7 @@ struct GemvOp {
     int bits;                    // code bytes per tile superstep = 512 * bits
     const uint16_t* x;           // fp16 [batch][k_in]
     uint16_t* y;                 // fp16 [batch][n_out]
-    float* partial;              // split-K partial sums (unused when n_chunks == 1)
-    unsigned* tile_count;        // split-K arrival counters, one per row pair
+    unsigned long long* partial; // split-K partial sums, one tagged word per (row pair, chunk, row, batch entry)
     int n_out, k_in;
     int n_ss, n_kb;              // supersteps, k blobs
     int n_rp;                    // row pairs = units per K chunk
@@ -72,6 +71,7 @@ struct Ctx {
     char* gemm_ws = nullptr;
     size_t gemm_ws_bytes = 0;
     uint64_t config_epoch = 0;
+    unsigned launch_epoch = 0;   // tag of the split-K partials of the latest decode launch (never 0)
     uint64_t stack_key = 0;      // hash of the op list that is currently uploaded
     bool stack_valid = false;
 };
@@ -93,9 +93,9 @@ int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, 
 
 // Chunking policy of the decode kernel: k blobs (512 columns) per K chunk.
 int gemv_chunk_blobs(int bits, int batch);
-size_t gemv_partial_floats_per_unit(int batch);
+size_t gemv_partial_bytes_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
-int launch_gemv_static(Ctx* ctx, GemvOp op, size_t counter_bytes, size_t partial_bytes, cudaStream_t st);
+int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st);
 // table_dev: [GemvOp x n_ops][long long phase_total x max(n_phases,1)][int cta_units x sm_count]
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
 // Units of an op (n_units units, block rotation rot) that CTA `cta` of `grid` processes: [lo, hi).

@@ -43,7 +43,7 @@ def test_static_scratch_gemv_matches_fq_gemv_twice():
 
 def test_static_scratch_gemv_rejects_oversized_layer():
     import paper_2501_07139_b200 as P
-    n, k = 32768, 8192                 # 2048 row tiles x 8 chunks x 64 B > 1 MiB of scratch
+    n, k = 32768, 8192                 # 1024 row pairs x 16 chunks x 256 B = 4 MiB > the built-in 2 MiB
     fq = P.FlexQ(1)
     codes = torch.zeros((n, k), dtype=torch.uint8, device="cuda")
     s = torch.ones((n, k // 128), dtype=torch.float16, device="cuda")
