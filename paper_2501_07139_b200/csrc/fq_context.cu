@@ -59,6 +59,7 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     }
     op.n_fields = fl.n;
     op.bits = bits;
+    op.variant = variant_index(L.fmt == FQ_FMT_PLANES, bits);
     op.store = static_cast<const uint8_t*>(v->store);
     op.blob_stride = blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits);
     op.blob_read = blob_bytes(bits);

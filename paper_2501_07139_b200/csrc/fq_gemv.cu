@@ -268,35 +268,67 @@ struct OpFetch {
 };
 static_assert(sizeof(GemvOp) <= 256, "op descriptor too large for the two-word fetch");
 
-// ------------------------------------------------------------------------------- one field, one superstep
-// Consumes field width F of TILES row tiles for one superstep: eight k32 steps, the first four
-// belong to the first group of 128 columns, the last four to the second.  Adds, per tile / pass / row /
-// group, the integer  2^shift * sum_k field_k * x_int_k  into v.
-//   MAXB == 1 : B columns (2t, 2t+1) carry the digits for bit-offset class t, lane (g, c) ends up with
-//               the partial sum of class c (still scaled by 2^(c*F)); xp[t] points at this lane's B
-//               data for class t (or at zeros).
-//   MAXB  > 1 : every register is shifted down to class 0; B columns (2b, 2b+1) carry batch entry
-//               4*pass + b; xp[pass] points at this lane's B data.
-// With one tile per warp the k32 steps of a group alternate between two accumulators, so that two
-// independent mma chains are in flight.
-template <int F, int MAXB, int TILES>
-__device__ __forceinline__ void field_step(const uint8_t* f0, bool two_pass, int lane, const uint8_t* const (&xp)[4],
-                                           int xoff, int shift, int (&v)[TILES][2][2][2])
+// ------------------------------------------------------------------------------- the arithmetic of one unit
+// Shared memory is addressed with 32-bit shared-window addresses and explicit ld.shared: the inner
+// loops then carry no 64-bit pointer arithmetic.
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+// D = A(u8, 16x32, row) * B(s8, 32x8, col): first link of an accumulation chain (C = 0).
+__device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+
+#ifndef FQ_GEMV_NA
+#define FQ_GEMV_NA 1
+#endif
+
+// One field of width F (at bit SHIFT of the code) of TILES row tiles, one superstep: eight k32 steps, the
+// first four belong to the first group of 128 columns, the last four to the second.  Adds (FIRSTF: stores),
+// per tile / pass / row / group, the integer  2^SHIFT * sum_k field_k * x_int_k  into v.
+//   fa     : shared address of this lane's 16-byte chunk in the first tile's field array
+//   MAXB 1 : B columns (2t, 2t+1) carry the activation digits for bit-offset class t; lane (g, c) ends up
+//            with the partial sum of class c, still scaled by 2^(c*F); xa[t] is the shared address of this
+//            lane's B data for class t (or of zeros)
+//   MAXB 8 : every register is shifted down to class 0; B columns (2b, 2b+1) carry batch entry
+//            4*pass + b; xa[pass] is this lane's B data
+// With one tile per warp and batch 1 the k32 steps of a group may alternate between FQ_GEMV_NA accumulators.
+template <int F, int SHIFT, bool FIRSTF, int MAXB, int TILES>
+__device__ __forceinline__ void field_step(uint32_t fa, const uint32_t (&xa)[4], uint32_t xoff, bool two_pass, int c,
+                                           int (&v)[TILES][MAXB == 1 ? 1 : 2][2][2])
 {
     constexpr int P = 8 / F;                                   // A registers stacked in one word
     constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
     constexpr int NP = MAXB == 1 ? 1 : 2;
-    constexpr int NA = (TILES == 1 && MAXB == 1) ? 2 : 1;      // accumulators per (tile, pass, group)
+    constexpr int NA = (TILES == 1 && MAXB == 1) ? FQ_GEMV_NA : 1;   // accumulators per (tile, pass, group)
     int acc[TILES][NP][2][NA][4];
-#pragma unroll
-    for (int i = 0; i < TILES * NP * 2 * NA * 4; i++) (&acc[0][0][0][0][0])[i] = 0;
 
 #pragma unroll
     for (int jb = 0; jb < F; jb++) {
         uint4 w[TILES], h[TILES];
 #pragma unroll
         for (int tl = 0; tl < TILES; tl++) {
-            w[tl] = *reinterpret_cast<const uint4*>(f0 + tl * F * 512 + jb * 512 + lane * 16);
+            w[tl] = lds128(fa + tl * F * 512 + jb * 512);
             h[tl] = w[tl];                                     // F == 1: classes 4..7 come down by one shift
             if (F == 1 && MAXB == 1) h[tl] = make_uint4(w[tl].x >> 4, w[tl].y >> 4, w[tl].z >> 4, w[tl].w >> 4);
         }
@@ -304,34 +336,50 @@ __device__ __forceinline__ void field_step(const uint8_t* f0, bool two_pass, int
         for (int t = 0; t < P; t++) {
             const int j = P * jb + t;                          // k32 step inside the superstep
             const int grp = j >> 2;
-            const int ai = NA == 2 ? (j & 1) : 0;
+            const int ai = (j & 3) % NA;
+            const bool first = (j & 3) < NA;                   // first link of this accumulator's chain
             if (MAXB == 1) {
                 const int tc = (F == 1) ? (t & 3) : t;         // bit-offset class = B column pair
                 const uint32_t m = kMask << (tc * F);
-                const uint2 x = *reinterpret_cast<const uint2*>(xp[tc] + xoff + j * 32);
+                const uint2 x = lds64(xa[tc] + xoff + j * 32);
 #pragma unroll
                 for (int tl = 0; tl < TILES; tl++) {
                     const uint4& a = (F == 1 && t >= 4) ? h[tl] : w[tl];
-                    mma_u8s8(acc[tl][0][grp][ai], a.x & m, a.y & m, a.z & m, a.w & m, x.x, x.y);
+                    if (F == 8) {
+                        if (first) mma_u8s8_first(acc[tl][0][grp][ai], a.x, a.y, a.z, a.w, x.x, x.y);
+                        else mma_u8s8(acc[tl][0][grp][ai], a.x, a.y, a.z, a.w, x.x, x.y);
+                    } else {
+                        if (first) mma_u8s8_first(acc[tl][0][grp][ai], a.x & m, a.y & m, a.z & m, a.w & m, x.x, x.y);
+                        else mma_u8s8(acc[tl][0][grp][ai], a.x & m, a.y & m, a.z & m, a.w & m, x.x, x.y);
+                    }
                 }
             } else {
                 const int sh = t * F;
-                const uint2 x = *reinterpret_cast<const uint2*>(xp[0] + xoff + j * 32);
+                const uint2 x = lds64(xa[0] + xoff + j * 32);
                 uint2 x2 = make_uint2(0u, 0u);
-                if (two_pass) x2 = *reinterpret_cast<const uint2*>(xp[1] + xoff + j * 32);
+                if (two_pass) x2 = lds64(xa[1] + xoff + j * 32);
 #pragma unroll
                 for (int tl = 0; tl < TILES; tl++) {
                     const uint32_t a0 = (w[tl].x >> sh) & kMask, a1 = (w[tl].y >> sh) & kMask;
                     const uint32_t a2 = (w[tl].z >> sh) & kMask, a3 = (w[tl].w >> sh) & kMask;
-                    mma_u8s8(acc[tl][0][grp][0], a0, a1, a2, a3, x.x, x.y);
-                    if (two_pass) mma_u8s8(acc[tl][NP - 1][grp][0], a0, a1, a2, a3, x2.x, x2.y);
+                    if (first) {
+                        mma_u8s8_first(acc[tl][0][grp][0], a0, a1, a2, a3, x.x, x.y);
+                        if (two_pass) mma_u8s8_first(acc[tl][NP - 1][grp][0], a0, a1, a2, a3, x2.x, x2.y);
+                        else if (NP > 1) {
+#pragma unroll
+                            for (int i = 0; i < 4; i++) acc[tl][NP - 1][grp][0][i] = 0;
+                        }
+                    } else {
+                        mma_u8s8(acc[tl][0][grp][0], a0, a1, a2, a3, x.x, x.y);
+                        if (two_pass) mma_u8s8(acc[tl][NP - 1][grp][0], a0, a1, a2, a3, x2.x, x2.y);
+                    }
                 }
             }
         }
     }
     // digits -> integer, undo the class scaling (exact: every term is a multiple of 2^(c*F)),
     // apply the field's position inside the code
-    const int down = MAXB == 1 ? (lane & 3) * F : 0;
+    const int down = MAXB == 1 ? c * F : 0;
 #pragma unroll
     for (int tl = 0; tl < TILES; tl++)
 #pragma unroll
@@ -340,10 +388,138 @@ __device__ __forceinline__ void field_step(const uint8_t* f0, bool two_pass, int
             for (int grp = 0; grp < 2; grp++) {
                 int a[4];
 #pragma unroll
-                for (int i = 0; i < 4; i++) a[i] = acc[tl][p][grp][0][i] + (NA == 2 ? acc[tl][p][grp][NA - 1][i] : 0);
-                v[tl][p][0][grp] += ((a[0] + (a[1] << 8)) >> down) << shift;
-                v[tl][p][1][grp] += ((a[2] + (a[3] << 8)) >> down) << shift;
+                for (int i = 0; i < 4; i++) {
+                    a[i] = acc[tl][p][grp][0][i];
+#pragma unroll
+                    for (int n = 1; n < NA; n++) a[i] += acc[tl][p][grp][n][i];
+                }
+                const int v0 = ((a[0] + (a[1] << 8)) >> down) << SHIFT, v1 = ((a[2] + (a[3] << 8)) >> down) << SHIFT;
+                if (FIRSTF) { v[tl][p][0][grp] = v0; v[tl][p][1][grp] = v1; }      // the first field starts the sums
+                else { v[tl][p][0][grp] += v0; v[tl][p][1][grp] += v1; }
             }
+}
+
+// The fields of one superstep, unrolled at compile time from the variant's field list.
+template <int VARIANT, int FI, int PREFIX, int MAXB, int TILES>
+struct FieldLoop {
+    static __device__ __forceinline__ void run(uint32_t fbase, int st_tile, const uint32_t (&xa)[4], uint32_t xoff,
+                                               bool two_pass, int c, int (&v)[TILES][MAXB == 1 ? 1 : 2][2][2])
+    {
+        constexpr FieldList FL = variant_fields(VARIANT);
+        if constexpr (FI < FL.n) {
+            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
+            // field array of width F after fields adding up to PREFIX bits; tile (superstep, row tile) = st_tile
+            const uint32_t fa = fbase + kBlobSteps * kBlobTiles * 512 * PREFIX + st_tile * (F * 512);
+            field_step<F, SHIFT, FI == 0, MAXB, TILES>(fa, xa, xoff, two_pass, c, v);
+            FieldLoop<VARIANT, FI + 1, PREFIX + F, MAXB, TILES>::run(fbase, st_tile, xa, xoff, two_pass, c, v);
+        }
+    }
+};
+
+// All supersteps of one unit for this warp's row tiles: tot[tile][pass][row half] += the dequantised dot products.
+//   st    : shared address of the stage          cnt : supersteps in the unit (whole blobs)
+//   xs    : shared address of the activation slot (digits, group sums, group scales)
+template <int VARIANT, int MAXB, int TILES, class S>
+__device__ __forceinline__ void unit_compute(uint32_t st, int cnt, int blob_read, uint32_t xs, uint32_t zero_page,
+                                             int B, int lane, int tile0, float (&tot)[TILES][MAXB == 1 ? 1 : 2][2])
+{
+    constexpr int NP = MAXB == 1 ? 1 : 2;
+    // a nested child reads the parent's top bits; the dropped bits are filled with their mid-point, which
+    // is the same as lowering every zero point by that amount
+    constexpr int kAdjust = (VARIANT >= 7 && VARIANT < 13) ? 1 << (7 - (VARIANT - 5)) : 0;
+    const int g = lane >> 2, c = lane & 3;
+    const bool two_pass = MAXB > 1 && B > 4;
+    // this lane's B-operand sources.  B column n = g holds digit (g & 1) of
+    //   batch 1: bit-offset class g >> 1            batch > 1: batch entry 4 * pass + (g >> 1)
+    uint32_t xa[4];
+    if (MAXB == 1) {
+#pragma unroll
+        for (int t = 0; t < 4; t++) xa[t] = (g >> 1) == t ? xs + (g & 1) * S::kDigitOff + c * 8 : zero_page + c * 8;
+    } else {
+#pragma unroll
+        for (int p = 0; p < 2; p++) {
+            const int b = 4 * p + (g >> 1);
+            xa[p] = b < B ? xs + b * S::kXRow + (g & 1) * S::kDigitOff + c * 8 : zero_page + c * 8;
+        }
+        xa[2] = xa[3] = zero_page + c * 8;
+    }
+    const uint32_t xsum = xs + S::kXsumOff, xscale = xs + S::kXscaleOff;
+    uint32_t blob = st;
+    for (int s = 0; s < cnt; s += kBlobSteps, blob += blob_read) {
+#ifdef FQ_GEMV_UNROLL_SSL
+#pragma unroll
+#else
+#pragma unroll 1                                                             // (keeps the 14 specialised loops small)
+#endif
+        for (int ssl = 0; ssl < kBlobSteps; ssl++) {
+            const int st_tile = ssl * kBlobTiles + tile0;
+            int v[TILES][NP][2][2];
+            FieldLoop<VARIANT, 0, 0, MAXB, TILES>::run(blob + kBlobMetaBytes + lane * 16, st_tile, xa, (s + ssl) * 256, two_pass, c, v);
+            // group epilogue: y += s * 2^-e * (v - z * sum x_int)
+            const uint32_t meta = blob + st_tile * 128 + g * 4;
+            if constexpr (MAXB == 1) {
+                // both groups' activation sums and scales in one load each; only the class-0 lane of a quad
+                // subtracts the zero-point term
+                const uint2 xs2 = lds64(xsum + (s + ssl) * 8), sc2 = lds64(xscale + (s + ssl) * 8);
+                const int nx[2] = {c == 0 ? -(int)xs2.x : 0, c == 0 ? -(int)xs2.y : 0};
+                const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
+#pragma unroll
+                for (int tl = 0; tl < TILES; tl++) {
+#pragma unroll
+                    for (int grp = 0; grp < 2; grp++) {
+                        const uint32_t m0 = lds32(meta + tl * 128 + grp * 64);
+                        const uint32_t m1 = lds32(meta + tl * 128 + grp * 64 + 32);
+                        const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
+                        const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
+                        // v - (z - adjust) * X  =  v + z * (-X) - adjust * (-X)
+                        const int base = kAdjust ? -kAdjust * nx[grp] : 0;
+                        const int t0 = v[tl][0][0][grp] + (int)(m0 >> 16) * nx[grp] + base;
+                        const int t1 = v[tl][0][1][grp] + (int)(m1 >> 16) * nx[grp] + base;
+                        tot[tl][0][0] = fmaf((float)t0, s0 * sc[grp], tot[tl][0][0]);
+                        tot[tl][0][1] = fmaf((float)t1, s1 * sc[grp], tot[tl][0][1]);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int tl = 0; tl < TILES; tl++) {
+#pragma unroll
+                    for (int grp = 0; grp < 2; grp++) {
+                        const uint32_t m0 = lds32(meta + tl * 128 + grp * 64);
+                        const uint32_t m1 = lds32(meta + tl * 128 + grp * 64 + 32);
+                        const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
+                        const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
+                        const int z0 = (int)(m0 >> 16) - kAdjust;
+                        const int z1 = (int)(m1 >> 16) - kAdjust;
+#pragma unroll
+                        for (int p = 0; p < NP; p++) {
+                            const int b = 4 * p + c;
+                            const bool has = b < B;
+                            const uint32_t gi = (uint32_t)(b * (S::kCMax * 2) + (s + ssl) * 2 + grp) * 4u;
+                            const int xsm = has ? (int)lds32(xsum + gi) : 0;
+                            const float scb = has ? __uint_as_float(lds32(xscale + gi)) : 0.f;
+                            tot[tl][p][0] = fmaf((float)(v[tl][p][0][grp] - z0 * xsm), s0 * scb, tot[tl][p][0]);
+                            tot[tl][p][1] = fmaf((float)(v[tl][p][1][grp] - z1 * xsm), s1 * scb, tot[tl][p][1]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int MAXB, int TILES, class S>
+__device__ __forceinline__ void unit_dispatch(int variant, uint32_t st, int cnt, int blob_read, uint32_t xs, uint32_t zero_page,
+                                              int B, int lane, int tile0, float (&tot)[TILES][MAXB == 1 ? 1 : 2][2])
+{
+#define FQ_VARIANT_CASE(V) case V: unit_compute<V, MAXB, TILES, S>(st, cnt, blob_read, xs, zero_page, B, lane, tile0, tot); break;
+    switch (variant) {
+        FQ_VARIANT_CASE(0) FQ_VARIANT_CASE(1) FQ_VARIANT_CASE(2) FQ_VARIANT_CASE(3) FQ_VARIANT_CASE(4)
+        FQ_VARIANT_CASE(5) FQ_VARIANT_CASE(6) FQ_VARIANT_CASE(7) FQ_VARIANT_CASE(8) FQ_VARIANT_CASE(9)
+        FQ_VARIANT_CASE(10) FQ_VARIANT_CASE(11) FQ_VARIANT_CASE(12) FQ_VARIANT_CASE(13)
+        default: break;
+    }
+#undef FQ_VARIANT_CASE
+    static_assert(kVariants == 14, "one case per variant");
 }
 
 template <int MAXB>
@@ -645,16 +821,17 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                         const int e = lane + 32 * i;                     // e = local row * BW + batch entry
                         const unsigned long long* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW) + e;
                         float acc = 0.f;
-                        for (int q0 = 0; q0 < d.n_chunks; q0 += 8) {
-                            unsigned long long w[8];
+                        constexpr int kLoads = MAXB == 1 ? 24 : 8;   // loads in flight: one round trip for most shapes
+                        for (int q0 = 0; q0 < d.n_chunks; q0 += kLoads) {
+                            unsigned long long w[kLoads];
 #pragma unroll
-                            for (int j = 0; j < 8; j++) {
+                            for (int j = 0; j < kLoads; j++) {
                                 const int q = q0 + j;
                                 w[j] = 0ull;
                                 if (q < d.n_chunks && q != d.ch) w[j] = ld_relaxed_u64(pt + (long long)q * (32 * BW));
                             }
 #pragma unroll
-                            for (int j = 0; j < 8; j++) {
+                            for (int j = 0; j < kLoads; j++) {
                                 const int q = q0 + j;
                                 if (q >= d.n_chunks) break;
                                 if (q == d.ch) acc += o[e];
@@ -706,7 +883,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 }
             }
             if (__shfl_sync(0xffffffffu, leave, 0)) break;
-            __nanosleep(m ? 100 : 32);
+            __nanosleep(20);
         }
     } else {
         // ================================================================== consumers
@@ -715,7 +892,6 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
         const int uidx = warp / kWarpsPerUnit;                       // which of the units in flight
         const int tile0 = (warp % kWarpsPerUnit) * kTilesPerWarp;    // first row tile of this warp
         constexpr int TL = kTilesPerWarp;
-        const uint8_t* zero_page = smem + S::oZero + c * 8;
         int total = 0;                               // units of this CTA over the whole launch
         if (sa.cta_units) total = sa.cta_units[cta];
         else {
@@ -727,38 +903,34 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
         float* odata = reinterpret_cast<float*>(smem + S::oOutData);
         OutDesc* odesc = reinterpret_cast<OutDesc*>(smem + S::oOutDesc);
         bool stop = false;
+        // ring position of this warp's next unit, advanced by additions
+        int stage = uidx % S::kStages;
+        unsigned use = (unsigned)(uidx / S::kStages);
+        const uint32_t opring_a = smem_u32(smem + S::oOpRing), desc_a = smem_u32(smem + S::oDesc);
         for (int seq = uidx; seq < total && !stop; seq += kUnitsInFlight) {
-            if (flags[1]) { stop = true; break; }
-            const int stage = seq % S::kStages;
-            const unsigned use = (unsigned)(seq / S::kStages);
             const uint32_t full = bars + 8 * stage, empty = bars + 8 * (S::kStages + stage);
             // a stage's uses are consumed strictly in order: wait for the release of the previous
             // use before trusting the parity of the full barrier
             bool ok = true;
             if (use > 0) ok = smem_wait([&] { return released[stage] >= use * kWarpsPerUnit || flags[1]; });
-            if (ok && !flags[1]) ok = mbar_wait(full, use & 1u);
+            if (ok) ok = mbar_wait(full, use & 1u);
             if (!ok || flags[1]) {
                 if (lane == 0 && !ok) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1; }
                 stop = true;
                 break;
             }
-            // (field widths and shifts travel as packed nibbles: a byte array indexed in the loop below
-            // would live in local memory)
-            struct { int ch, rp, cnt, seg, blob_read, n_fields, zero_adjust, batch, op_slot, oseq, n_chunks;
-                     unsigned long long* partial; uint32_t widths, shifts; } d;
+            struct { int ch, rp, cnt, seg, blob_read, variant, batch, op_slot, oseq, n_chunks;
+                     unsigned long long* partial; } d;
             {
-                const UnitDesc ud = *(reinterpret_cast<const UnitDesc*>(smem + S::oDesc) + stage);
-                const GemvOp& od = *reinterpret_cast<const GemvOp*>(opring + ud.op_slot * S::kOpBytes);
-                d.ch = ud.ch; d.rp = ud.rp; d.cnt = ud.nb * kBlobSteps; d.seg = ud.seg; d.op_slot = ud.op_slot;
-                d.blob_read = od.blob_read; d.n_fields = od.n_fields;
-                d.zero_adjust = od.zero_adjust; d.batch = od.batch;
-                d.oseq = ud.oseq; d.n_chunks = od.n_chunks; d.partial = od.partial;
-                d.widths = 0u; d.shifts = 0u;
-#pragma unroll
-                for (int i = 0; i < kMaxFields; i++) {
-                    d.widths |= (uint32_t)od.field_width[i] << (4 * i);
-                    d.shifts |= (uint32_t)od.field_shift[i] << (4 * i);
-                }
+                const uint4 u0 = lds128(desc_a + stage * (int)sizeof(UnitDesc));            // ch, rp, nb, seg
+                const uint2 u1 = lds64(desc_a + stage * (int)sizeof(UnitDesc) + 16);        // op_slot, oseq
+                const uint32_t od = opring_a + u1.x * S::kOpBytes;
+                const uint4 o1 = lds128(od + 16);                                           // blob_read, variant, batch, n_chunks
+                const uint2 o0 = lds64(od + 8);                                             // partial
+                d.ch = (int)u0.x; d.rp = (int)u0.y; d.cnt = (int)u0.z * kBlobSteps; d.seg = (int)u0.w;
+                d.op_slot = (int)u1.x; d.oseq = (int)u1.y;
+                d.blob_read = (int)o1.x; d.variant = (int)o1.y; d.batch = (int)o1.z; d.n_chunks = (int)o1.w;
+                d.partial = reinterpret_cast<unsigned long long*>(((unsigned long long)o0.y << 32) | o0.x);
             }
             // a unit that finishes its row pair needs a place in the output queue: that place must be free
             // again; the descriptor goes there now, while the op's slot in the op ring is certainly still valid
@@ -778,7 +950,6 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     q.y = od.y; q.partial = od.partial;
                 }
             }
-            const uint8_t* st = smem + S::oStages + stage * S::kStageBytes;
             const int slot = d.seg % kXSlots;
             if (!smem_wait([&] { return x_ready[slot] == d.seg + 1 || flags[1]; })) {
                 if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; }
@@ -786,76 +957,15 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
             __threadfence_block();
             __syncwarp();
             const bool live = !flags[0];
-            const int B = d.batch;
-            const bool two_pass = MAXB > 1 && B > 4;
-            const uint8_t* xs = smem + S::oX + slot * S::kXSlotBytes;
 
             float tot[TL][NP][2];
 #pragma unroll
             for (int i = 0; i < TL * NP * 2; i++) (&tot[0][0][0])[i] = 0.f;
 
-            if (live) {
-                // this lane's B-operand sources.  B column n = g holds digit (g & 1) of
-                //   batch 1: bit-offset class g >> 1            batch > 1: batch entry 4 * pass + (g >> 1)
-                const uint8_t* xp[4];
-                if (MAXB == 1) {
-#pragma unroll
-                    for (int t = 0; t < 4; t++)
-                        xp[t] = (g >> 1) == t ? xs + (g & 1) * S::kDigitOff + c * 8 : zero_page;
-                } else {
-#pragma unroll
-                    for (int p = 0; p < 2; p++) {
-                        const int b = 4 * p + (g >> 1);
-                        xp[p] = b < B ? xs + b * S::kXRow + (g & 1) * S::kDigitOff + c * 8 : zero_page;
-                    }
-                    xp[2] = zero_page; xp[3] = zero_page;
-                }
-                const int* xsum = reinterpret_cast<const int*>(xs + S::kXsumOff);
-                const float* xscale = reinterpret_cast<const float*>(xs + S::kXscaleOff);
-                for (int s = 0; s < d.cnt; s++) {
-                    const uint8_t* blob = st + (s / kBlobSteps) * d.blob_read;       // this superstep's blob (prefix)
-                    const int ssl = s % kBlobSteps;
-                    const uint32_t* meta_s = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile0));
-                    int v[TL][2][2][2];
-#pragma unroll
-                    for (int i = 0; i < TL * 8; i++) (&v[0][0][0][0])[i] = 0;
-                    int prefix = 0;
-                    for (int fi = 0; fi < d.n_fields; fi++) {
-                        const int f = (d.widths >> (4 * fi)) & 15, fshift = (d.shifts >> (4 * fi)) & 15;
-                        const uint8_t* f0 = blob + blob_field_off(prefix, f, ssl, tile0);
-                        switch (f) {
-                            case 8: field_step<8, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
-                            case 4: field_step<4, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
-                            case 2: field_step<2, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
-                            default: field_step<1, MAXB, TL>(f0, two_pass, lane, xp, s * 256, fshift, v); break;
-                        }
-                        prefix += f;
-                    }
-                    // group epilogue: y += s * 2^-e * (v - z * sum x_int)
-#pragma unroll
-                    for (int tl = 0; tl < TL; tl++) {
-#pragma unroll
-                        for (int grp = 0; grp < 2; grp++) {
-                            const uint32_t m0 = meta_s[tl * 32 + grp * 16 + g];
-                            const uint32_t m1 = meta_s[tl * 32 + grp * 16 + g + 8];
-                            const float s0 = __half2float(__ushort_as_half((unsigned short)(m0 & 0xffffu)));
-                            const float s1 = __half2float(__ushort_as_half((unsigned short)(m1 & 0xffffu)));
-                            const int z0 = (int)(m0 >> 16) - d.zero_adjust;
-                            const int z1 = (int)(m1 >> 16) - d.zero_adjust;
-#pragma unroll
-                            for (int p = 0; p < NP; p++) {
-                                // batch 1: only the class-0 lane subtracts the zero-point term
-                                const int b = MAXB == 1 ? 0 : 4 * p + c;
-                                const bool has = MAXB == 1 ? true : b < B;
-                                const int xsm = (MAXB == 1 ? c == 0 : has) ? xsum[b * (S::kCMax * 2) + s * 2 + grp] : 0;
-                                const float sc = has ? xscale[b * (S::kCMax * 2) + s * 2 + grp] : 0.f;
-                                tot[tl][p][0] = fmaf((float)(v[tl][p][0][grp] - z0 * xsm), s0 * sc, tot[tl][p][0]);
-                                tot[tl][p][1] = fmaf((float)(v[tl][p][1][grp] - z1 * xsm), s1 * sc, tot[tl][p][1]);
-                            }
-                        }
-                    }
-                }
-            }
+            if (live)
+                unit_dispatch<MAXB, TL, S>(d.variant, smem_u32(smem + S::oStages) + (uint32_t)stage * S::kStageBytes, d.cnt,
+                                           d.blob_read, smem_u32(smem + S::oX) + (uint32_t)slot * S::kXSlotBytes,
+                                           smem_u32(smem + S::oZero), d.batch, lane, tile0, tot);
             __syncwarp();
             if (lane == 0) {
                 atomicAdd(const_cast<unsigned*>(&released[stage]), 1u);
@@ -863,6 +973,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 mbar_arrive(empty);                              // the stage may be refilled
                 atomicSub(const_cast<int*>(&x_pending[slot]), 1);   // one warp fewer needs the activation slot
             }
+            stage += kUnitsInFlight;
+            while (stage >= S::kStages) { stage -= S::kStages; use++; }
             if (!live) continue;
 
             if (MAXB == 1) {                                     // add up the bit-offset classes held by the quad

@@ -1,6 +1,7 @@
 // Host-side context and the descriptors passed to the kernels.
 #pragma once
 #include <cuda_runtime.h>
+#include <cstddef>
 #include <cstdint>
 #include <vector>
 
@@ -27,26 +28,29 @@ constexpr int kUnitRowTiles = 2;   // a decode unit covers two 16-row tiles (32 
 // What one decode op needs on the device.
 struct GemvOp {
     const uint8_t* store;        // blobs [row_pair][k_blob]
-    int blob_stride;             // bytes from one blob to the next (size of the stored variant's blobs)
+    unsigned long long* partial; // split-K partial sums, one tagged word per (row pair, chunk, row, batch entry)
+    // read by every consumer warp for every unit: kept together, 16-byte aligned, one vector load
     int blob_read;               // bytes of every blob that this op reads (all of it, or a nested child's prefix)
-    uint8_t field_width[kMaxFields];
-    uint8_t field_shift[kMaxFields];
-    int n_fields;
-    int bits;                    // code bytes per tile superstep = 512 * bits
+    int variant;                 // variant_index(format, bits): selects the specialised inner loop
+    int batch;
+    int n_chunks;                // K chunks
     const uint16_t* x;           // fp16 [batch][k_in]
     uint16_t* y;                 // fp16 [batch][n_out]
-    unsigned long long* partial; // split-K partial sums, one tagged word per (row pair, chunk, row, batch entry)
+    int blob_stride;             // bytes from one blob to the next (size of the stored variant's blobs)
+    int n_fields;
+    uint8_t field_width[kMaxFields];
+    uint8_t field_shift[kMaxFields];
+    int bits;                    // code bytes per tile superstep = 512 * bits
     int n_out, k_in;
     int n_ss, n_kb;              // supersteps, k blobs
     int n_rp;                    // row pairs = units per K chunk
-    int n_chunks;                // K chunks
     int chunk_blobs;             // k blobs per K chunk (the last chunk may be shorter)
-    int batch;
     int zero_adjust;             // subtracted from every zero point (mid-point fill of a nested child)
     int phase;                   // -1: no ordering
     int n_units;                 // n_chunks * n_rp
     int rot;                     // rotation of the CTA blocks for this op (evens out remainders)
 };
+static_assert(offsetof(GemvOp, blob_read) == 16 && offsetof(GemvOp, partial) == 8, "consumer block of the op descriptor");
 
 struct StackHeader {
     int n_ops;

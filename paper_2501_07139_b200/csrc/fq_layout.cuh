@@ -30,6 +30,7 @@
 #else
 #define FQ_HD inline
 #endif
+#define FQ_HDC constexpr FQ_HD
 
 namespace fq {
 
@@ -45,7 +46,7 @@ struct FieldList {
 };
 
 // Fields of a PACKED variant of `bits` bits (most significant first).
-FQ_HD FieldList packed_fields(int bits)
+FQ_HDC FieldList packed_fields(int bits)
 {
     FieldList fl{};
     int rem = bits;
@@ -61,7 +62,7 @@ FQ_HD FieldList packed_fields(int bits)
 
 // Fields of the 8-bit PLANES parent restricted to its `bits` most significant bits.
 // Shifts are in parent code units.
-FQ_HD FieldList plane_fields(int bits)
+FQ_HDC FieldList plane_fields(int bits)
 {
     FieldList fl{};
     fl.width[0] = 2; fl.shift[0] = 6; fl.n = 1;
@@ -76,6 +77,12 @@ FQ_HD FieldList plane_fields(int bits)
 FQ_HD int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 FQ_HD int row_tiles(int n_out) { return (n_out + kTileRows - 1) / kTileRows; }
 FQ_HD int supersteps(int k_in) { return (k_in + kStepCols - 1) / kStepCols; }
+
+// Decode kernels are specialised per field list.  Variant index: 0..6 = PACKED 2..8 bits, 7..13 = a
+// 2..8-bit child of the PLANES parent.
+constexpr int kVariants = 14;
+FQ_HDC int variant_index(bool planes, int bits) { return (planes ? 7 : 0) + bits - 2; }
+FQ_HDC FieldList variant_fields(int variant) { return variant < 7 ? packed_fields(variant + 2) : plane_fields(variant - 5); }
 
 constexpr int kBlobSteps = 2;             // supersteps per blob
 constexpr int kBlobTiles = 2;             // row tiles per blob (a row pair)
