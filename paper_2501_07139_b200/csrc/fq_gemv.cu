@@ -53,13 +53,13 @@ constexpr int kOutputWarp = kPrepWarp + kPrepWarps;    // the warp that owns eve
 constexpr int kGemvThreads = (kConsumerWarps + 1 + kPrepWarps + 1) * 32;
 constexpr int kUnitBytes = FQ_GEMV_UNIT_BYTES;         // bytes of one unit (whole blobs), at most: 2 x 4-bit or 1 x 8-bit blob
 constexpr int kXSlots = 3;                             // activation chunks kept in shared memory
-constexpr int kOutSlots = 32;                          // finished units waiting for the output warp
-static_assert(kOutSlots <= 32, "the output warp scans one slot per lane");
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 template <int MAXB> struct GemvCfg;
-template <> struct GemvCfg<1> { static constexpr int kBlobsMax = 3; };  // k blobs (512 columns) per chunk, at most
-template <> struct GemvCfg<8> { static constexpr int kBlobsMax = 1; };
+// kBlobsMax: k blobs (512 columns) per chunk, at most.  kOutSlots: finished units waiting for the output
+// warp (it scans one slot per lane: at most 32).
+template <> struct GemvCfg<1> { static constexpr int kBlobsMax = 3, kOutSlots = 32; };
+template <> struct GemvCfg<8> { static constexpr int kBlobsMax = 2, kOutSlots = 16; };
 
 // What the producer tells the consumers: once per op a copy of the op descriptor in a ring ...
 constexpr int kOpRing = 16;                            // > stages + 1: an op slot outlives the start of its last unit
@@ -83,6 +83,7 @@ static_assert(sizeof(OutDesc) == 48, "descriptor layout");
 
 template <int MAXB> struct GemvSmem {
     static constexpr int kCMax = GemvCfg<MAXB>::kBlobsMax * kBlobSteps;     // supersteps per chunk, at most
+    static constexpr int kOutSlots = GemvCfg<MAXB>::kOutSlots;
     static constexpr int kStageBytes = kUnitBytes;
     // activation slot: low digits, high digits (rows padded so that LDS.64 of a quarter warp is
     // conflict free), then per (row, group) the integer sum and the power-of-two scale
@@ -537,8 +538,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
     volatile int* flags = x_pending + kXSlots;                                 // [0]: stop computing, [1]: stop everything
     volatile int* prep_cmd = flags + 2;                                        // decision shared by the pre-processing warps
     volatile unsigned* out_fill = reinterpret_cast<volatile unsigned*>(smem + S::oOutCtl);   // consumer warps that filled a slot
-    volatile unsigned* out_gen = out_fill + kOutSlots;                         // times the output warp drained a slot
-    volatile int* out_total = reinterpret_cast<volatile int*>(out_gen + kOutSlots);   // finishing units of this CTA (-1: not known yet)
+    volatile unsigned* out_gen = out_fill + S::kOutSlots;                         // times the output warp drained a slot
+    volatile int* out_total = reinterpret_cast<volatile int*>(out_gen + S::kOutSlots);   // finishing units of this CTA (-1: not known yet)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::kStages; s++) {
@@ -547,7 +548,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
             released[s] = 0u;
         }
         for (int i = 0; i < kXSlots; i++) { x_ready[i] = 0; x_pending[i] = 0; }
-        for (int i = 0; i < kOutSlots; i++) { out_fill[i] = 0u; out_gen[i] = 0u; }
+        for (int i = 0; i < S::kOutSlots; i++) { out_fill[i] = 0u; out_gen[i] = 0u; }
         out_total[0] = -1;
         flags[0] = 0; flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -805,7 +806,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
         unsigned idle_it = 0u;
         for (;;) {
             // every decision that ends the loop is taken by lane 0 and broadcast: the lanes must leave together
-            const bool filled = lane < kOutSlots && out_fill[lane] == (unsigned)kWarpsPerUnit;
+            const bool filled = lane < S::kOutSlots && out_fill[lane] == (unsigned)kWarpsPerUnit;
             const unsigned m = __ballot_sync(0xffffffffu, filled);
             unsigned done = 0u;
             if (m) {
@@ -814,34 +815,39 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     const int s = __ffs(mm) - 1;
                     const OutDesc& d = odesc[s];
                     const float* o = odata + s * S::kOutFloats;
+                    // a few chunks per round trip, every batch entry of them in flight at once; a round whose
+                    // words are not all there ends the attempt
+                    constexpr int QS = MAXB == 1 ? 24 : 2;
                     float sum[BW];
+#pragma unroll
+                    for (int i = 0; i < BW; i++) sum[i] = 0.f;
                     bool ok = true;
+                    const unsigned long long* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW) + lane;
+                    for (int q0 = 0; q0 < d.n_chunks; q0 += QS) {
+                        unsigned long long w[QS][BW];
 #pragma unroll
-                    for (int i = 0; i < BW; i++) {
-                        const int e = lane + 32 * i;                     // e = local row * BW + batch entry
-                        const unsigned long long* pt = d.partial + (long long)d.rp * d.n_chunks * (32 * BW) + e;
-                        float acc = 0.f;
-                        constexpr int kLoads = MAXB == 1 ? 24 : 8;   // loads in flight: one round trip for most shapes
-                        for (int q0 = 0; q0 < d.n_chunks; q0 += kLoads) {
-                            unsigned long long w[kLoads];
+                        for (int j = 0; j < QS; j++) {
+                            const int q = q0 + j;
 #pragma unroll
-                            for (int j = 0; j < kLoads; j++) {
-                                const int q = q0 + j;
-                                w[j] = 0ull;
-                                if (q < d.n_chunks && q != d.ch) w[j] = ld_relaxed_u64(pt + (long long)q * (32 * BW));
+                            for (int i = 0; i < BW; i++) {                // element e = lane + 32 i = local row * BW + batch entry
+                                w[j][i] = 0ull;
+                                if (q < d.n_chunks && q != d.ch) w[j][i] = ld_relaxed_u64(pt + (long long)q * (32 * BW) + 32 * i);
                             }
+                        }
 #pragma unroll
-                            for (int j = 0; j < kLoads; j++) {
-                                const int q = q0 + j;
-                                if (q >= d.n_chunks) break;
-                                if (q == d.ch) acc += o[e];
+                        for (int j = 0; j < QS; j++) {
+                            const int q = q0 + j;
+                            if (q >= d.n_chunks) break;
+#pragma unroll
+                            for (int i = 0; i < BW; i++) {
+                                if (q == d.ch) sum[i] += o[lane + 32 * i];
                                 else {
-                                    ok = ok && (unsigned)(w[j] >> 32) == sa.epoch;
-                                    acc += __uint_as_float((unsigned)w[j]);
+                                    ok = ok && (unsigned)(w[j][i] >> 32) == sa.epoch;
+                                    sum[i] += __uint_as_float((unsigned)w[j][i]);
                                 }
                             }
                         }
-                        sum[i] = acc;
+                        if (!__all_sync(0xffffffffu, ok)) break;
                     }
                     if (!__all_sync(0xffffffffu, ok)) continue;          // some chunk has not arrived yet: look again later
                     const int row_base = d.rp * (kUnitRowTiles * kTileRows);
@@ -934,9 +940,9 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
             }
             // a unit that finishes its row pair needs a place in the output queue: that place must be free
             // again; the descriptor goes there now, while the op's slot in the op ring is certainly still valid
-            const int oslot = d.oseq % kOutSlots;
+            const int oslot = d.oseq % S::kOutSlots;
             if (d.oseq >= 0) {
-                const unsigned ogen = (unsigned)(d.oseq / kOutSlots);
+                const unsigned ogen = (unsigned)(d.oseq / S::kOutSlots);
                 if (!smem_wait([&] { return out_gen[oslot] == ogen || flags[1]; })) {
                     if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; flags[1] = 1; }
                     stop = true;
