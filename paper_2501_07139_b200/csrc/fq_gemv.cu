@@ -25,6 +25,8 @@
 // computing, drains its copies and returns.
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "fq_internal.cuh"
 
 namespace fq {
@@ -113,10 +115,12 @@ template <int MAXB> struct GemvSmem {
     static constexpr int oReleased = oBars + 2 * kStages * 8;        // u32[S]: consumer warps that released a stage, ever
     static constexpr int oCtl = oReleased + kStages * 4;             // x_ready[XS], x_pending[XS], flags[2], prep_cmd, pad
     static constexpr int oOutCtl = oCtl + 64;                        // out_fill[kOutSlots], out_gen[kOutSlots]
-    static constexpr int kTotal = oOutCtl + 2 * kOutSlots * 4 + 16;  // + out_total
+    static constexpr int oXBars = (oOutCtl + 2 * kOutSlots * 4 + 16 + 7) / 8 * 8;   // (+ out_total) one mbarrier per activation slot
+    static constexpr int kTotal = oXBars + 8 * kXSlots + 8;
     static_assert(kStages >= 4, "decode kernel: no room for a ring");
     static_assert(kOpRing >= kStages + 2, "an op's ring slot must outlive the units that refer to it");
     static_assert(kTotal <= 232448, "decode kernel: shared memory over the 227 KB per-CTA limit");
+    static_assert(oBars % 8 == 0 && oXBars % 8 == 0, "mbarriers are 8-byte objects");
 };
 
 // K blobs (512 columns) per K chunk for a variant of which `bits` bits are read.
@@ -171,7 +175,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     const unsigned long long t0 = global_ns();
     for (;;) {
         for (int i = 0; i < 64; i++)
-            if (mbar_try_wait(bar, parity)) return true;
+            if (mbar_try_wait(bar, parity)) return true;      // (no back-off: a sleep here costs 20 % throughput)
         if (global_ns() - t0 > kWaitLimitNs) return false;
     }
 }
@@ -184,7 +188,7 @@ __device__ __forceinline__ bool smem_wait(Pred pred)
     for (;;) {
         for (int i = 0; i < 64; i++) {
             if (pred()) return true;
-            __nanosleep(20);
+            __nanosleep(20);                       // (a tight spin here takes issue slots from the consumers: -10 %)
         }
         if (global_ns() - t0 > kWaitLimitNs) return false;
     }
@@ -272,23 +276,36 @@ static_assert(sizeof(GemvOp) <= 256, "op descriptor too large for the two-word f
 // ------------------------------------------------------------------------------- the arithmetic of one unit
 // Shared memory is addressed with 32-bit shared-window addresses and explicit ld.shared: the inner
 // loops then carry no 64-bit pointer arithmetic.
+// (OFF is a compile-time byte offset: it goes into the instruction's address field instead of costing an add)
+template <int OFF = 0>
 __device__ __forceinline__ uint4 lds128(uint32_t a)
 {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a), "n"(OFF));
     return v;
 }
+template <int OFF = 0>
 __device__ __forceinline__ uint2 lds64(uint32_t a)
 {
     uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(a), "n"(OFF));
     return v;
 }
+template <int OFF = 0>
 __device__ __forceinline__ uint32_t lds32(uint32_t a)
 {
     uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF));
     return v;
+}
+// Loop whose index is a compile-time constant in the body (so that it can be a load's immediate offset).
+template <int I, int N, class Fn>
+__device__ __forceinline__ void static_for(Fn&& fn)
+{
+    if constexpr (I < N) {
+        fn(std::integral_constant<int, I>{});
+        static_for<I + 1, N>(fn);
+    }
 }
 // D = A(u8, 16x32, row) * B(s8, 32x8, col): first link of an accumulation chain (C = 0).
 __device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -324,25 +341,25 @@ __device__ __forceinline__ void field_step(uint32_t fa, const uint32_t (&xa)[4],
     constexpr int NA = (TILES == 1 && MAXB == 1) ? FQ_GEMV_NA : 1;   // accumulators per (tile, pass, group)
     int acc[TILES][NP][2][NA][4];
 
-#pragma unroll
-    for (int jb = 0; jb < F; jb++) {
+    static_for<0, F>([&](auto JB) {
+        constexpr int jb = decltype(JB)::value;
         uint4 w[TILES], h[TILES];
-#pragma unroll
-        for (int tl = 0; tl < TILES; tl++) {
-            w[tl] = lds128(fa + tl * F * 512 + jb * 512);
+        static_for<0, TILES>([&](auto TLI) {
+            constexpr int tl = decltype(TLI)::value;
+            w[tl] = lds128<tl * F * 512 + jb * 512>(fa);
             h[tl] = w[tl];                                     // F == 1: classes 4..7 come down by one shift
             if (F == 1 && MAXB == 1) h[tl] = make_uint4(w[tl].x >> 4, w[tl].y >> 4, w[tl].z >> 4, w[tl].w >> 4);
-        }
-#pragma unroll
-        for (int t = 0; t < P; t++) {
-            const int j = P * jb + t;                          // k32 step inside the superstep
-            const int grp = j >> 2;
-            const int ai = (j & 3) % NA;
-            const bool first = (j & 3) < NA;                   // first link of this accumulator's chain
-            if (MAXB == 1) {
-                const int tc = (F == 1) ? (t & 3) : t;         // bit-offset class = B column pair
-                const uint32_t m = kMask << (tc * F);
-                const uint2 x = lds64(xa[tc] + xoff + j * 32);
+        });
+        static_for<0, P>([&](auto TI) {
+            constexpr int t = decltype(TI)::value;
+            constexpr int j = P * jb + t;                      // k32 step inside the superstep
+            constexpr int grp = j >> 2;
+            [[maybe_unused]] constexpr int ai = (j & 3) % NA;
+            constexpr bool first = (j & 3) < NA;               // first link of this accumulator's chain
+            if constexpr (MAXB == 1) {
+                constexpr int tc = (F == 1) ? (t & 3) : t;     // bit-offset class = B column pair
+                constexpr uint32_t m = kMask << (tc * F);
+                const uint2 x = lds64<j * 32>(xa[tc] + xoff);
 #pragma unroll
                 for (int tl = 0; tl < TILES; tl++) {
                     const uint4& a = (F == 1 && t >= 4) ? h[tl] : w[tl];
@@ -355,10 +372,10 @@ __device__ __forceinline__ void field_step(uint32_t fa, const uint32_t (&xa)[4],
                     }
                 }
             } else {
-                const int sh = t * F;
-                const uint2 x = lds64(xa[0] + xoff + j * 32);
+                constexpr int sh = t * F;
+                const uint2 x = lds64<j * 32>(xa[0] + xoff);
                 uint2 x2 = make_uint2(0u, 0u);
-                if (two_pass) x2 = lds64(xa[1] + xoff + j * 32);
+                if (two_pass) x2 = lds64<j * 32>(xa[1] + xoff);
 #pragma unroll
                 for (int tl = 0; tl < TILES; tl++) {
                     const uint32_t a0 = (w[tl].x >> sh) & kMask, a1 = (w[tl].y >> sh) & kMask;
@@ -376,8 +393,8 @@ __device__ __forceinline__ void field_step(uint32_t fa, const uint32_t (&xa)[4],
                     }
                 }
             }
-        }
-    }
+        });
+    });
     // digits -> integer, undo the class scaling (exact: every term is a multiple of 2^(c*F)),
     // apply the field's position inside the code
     const int down = MAXB == 1 ? c * F : 0;
@@ -464,22 +481,19 @@ __device__ __forceinline__ void unit_compute(uint32_t st, int cnt, int blob_read
                 const uint2 xs2 = lds64(xsum + (s + ssl) * 8), sc2 = lds64(xscale + (s + ssl) * 8);
                 const int nx[2] = {c == 0 ? -(int)xs2.x : 0, c == 0 ? -(int)xs2.y : 0};
                 const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
-#pragma unroll
-                for (int tl = 0; tl < TILES; tl++) {
-#pragma unroll
-                    for (int grp = 0; grp < 2; grp++) {
-                        const uint32_t m0 = lds32(meta + tl * 128 + grp * 64);
-                        const uint32_t m1 = lds32(meta + tl * 128 + grp * 64 + 32);
-                        const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
-                        const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
-                        // v - (z - adjust) * X  =  v + z * (-X) - adjust * (-X)
-                        const int base = kAdjust ? -kAdjust * nx[grp] : 0;
-                        const int t0 = v[tl][0][0][grp] + (int)(m0 >> 16) * nx[grp] + base;
-                        const int t1 = v[tl][0][1][grp] + (int)(m1 >> 16) * nx[grp] + base;
-                        tot[tl][0][0] = fmaf((float)t0, s0 * sc[grp], tot[tl][0][0]);
-                        tot[tl][0][1] = fmaf((float)t1, s1 * sc[grp], tot[tl][0][1]);
-                    }
-                }
+                static_for<0, TILES * 2>([&](auto I) {
+                    constexpr int tl = decltype(I)::value / 2, grp = decltype(I)::value % 2;
+                    const uint32_t m0 = lds32<tl * 128 + grp * 64>(meta);
+                    const uint32_t m1 = lds32<tl * 128 + grp * 64 + 32>(meta);
+                    const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
+                    const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
+                    // v - (z - adjust) * X  =  v + z * (-X) - adjust * (-X)
+                    const int base = kAdjust ? -kAdjust * nx[grp] : 0;
+                    const int t0 = v[tl][0][0][grp] + (int)(m0 >> 16) * nx[grp] + base;
+                    const int t1 = v[tl][0][1][grp] + (int)(m1 >> 16) * nx[grp] + base;
+                    tot[tl][0][0] = fmaf((float)t0, s0 * sc[grp], tot[tl][0][0]);
+                    tot[tl][0][1] = fmaf((float)t1, s1 * sc[grp], tot[tl][0][1]);
+                });
             } else {
 #pragma unroll
                 for (int tl = 0; tl < TILES; tl++) {
@@ -534,6 +548,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
     const uint32_t bars = smem_u32(smem + S::oBars);                          // full[0..S), empty[0..S)
     volatile unsigned* released = reinterpret_cast<volatile unsigned*>(smem + S::oReleased);
     volatile int* x_ready = reinterpret_cast<volatile int*>(smem + S::oCtl);   // segment number + 1 held by a slot
+    const uint32_t xbars = smem_u32(smem + S::oXBars);                         // completes a phase per publication of a slot
     volatile int* x_pending = x_ready + kXSlots;                               // units that still need the slot
     volatile int* flags = x_pending + kXSlots;                                 // [0]: stop computing, [1]: stop everything
     volatile int* prep_cmd = flags + 2;                                        // decision shared by the pre-processing warps
@@ -547,7 +562,7 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
             mbar_init(bars + 8 * (S::kStages + s), kWarpsPerUnit);
             released[s] = 0u;
         }
-        for (int i = 0; i < kXSlots; i++) { x_ready[i] = 0; x_pending[i] = 0; }
+        for (int i = 0; i < kXSlots; i++) { x_ready[i] = 0; x_pending[i] = 0; mbar_init(xbars + 8 * i, 1); }
         for (int i = 0; i < S::kOutSlots; i++) { out_fill[i] = 0u; out_gen[i] = 0u; }
         out_total[0] = -1;
         flags[0] = 0; flags[1] = 0;
@@ -696,7 +711,6 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                         const unsigned long long t0 = global_ns();
                         unsigned it = 0;
                         while (ld_acquire_u64(sa.phase_done + (op.phase - 1)) < need) {
-                            __nanosleep(40);
                             if ((++it & 63u) == 0u &&
                                 (global_ns() - t0 > kWaitLimitNs || *reinterpret_cast<volatile int*>(sa.status) != 0 ||
                                  flags[0])) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; break; }
@@ -788,6 +802,8 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                     x_pending[slot] = units * kWarpsPerUnit;
                     __threadfence_block();
                     x_ready[slot] = seg + 1;
+                    __threadfence_block();
+                    mbar_arrive(xbars + 8 * slot);                     // wakes the consumers that sleep on this slot
                 }
             }
         }
@@ -957,6 +973,10 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                 }
             }
             const int slot = d.seg % kXSlots;
+            // sleep on the slot's barrier (a hardware wake-up: this wait is on the critical path of every
+            // dependency phase); the flag has the last word, because a warp that is several publications
+            // ahead would read a stale parity
+            if (x_ready[slot] != d.seg + 1 && !flags[1]) mbar_wait(xbars + 8 * slot, (unsigned)(d.seg / kXSlots) & 1u);
             if (!smem_wait([&] { return x_ready[slot] == d.seg + 1 || flags[1]; })) {
                 if (lane == 0) { atomicCAS(sa.status, 0, FQ_ERR_TIMEOUT); flags[0] = 1; }
             }
