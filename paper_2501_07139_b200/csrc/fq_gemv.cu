@@ -1,22 +1,28 @@
 // Decode path: fused dequantize-GEMV over tiled field arrays, batch 1..8.
 //
-// One persistent CTA per SM with three roles:
-//   producer thread : streams "units" (32 output rows x one K chunk: every field array of the
+// One persistent CTA per SM with four roles:
+//   producer warp   : streams "units" (32 output rows x one K chunk: every field array of the
 //                     active variant plus the scale/zero words) from HBM into a shared-memory
 //                     ring with bulk asynchronous copies (cp.async.bulk + mbarrier tx counts)
 //                     and writes a small descriptor next to each stage;
-//   x-prep warp     : once per (op, K chunk) that this CTA touches, waits -- bounded -- for the
-//                     previous dependency phase, loads the activations of that chunk and turns
+//   x-prep warps    : once per (op, K chunk) that this CTA touches, wait -- bounded -- for the
+//                     previous dependency phase, load the activations of that chunk and turn
 //                     them into 16-bit fixed point per group of 128 columns
 //                     (x_int = rint(x * 2^e), |x_int| < 2^14, stored as two signed byte digits);
-//   8 consumer warps: stored words become 8-bit mma.m16n8k32 A operands with ONE AND each (no
-//                     shift: a word holds 8/f registers on top of each other, see fq_layout.cuh),
-//                     the activation digits are the B operand, accumulation is exact in s32.
-//                     At batch 1 the eight B columns carry (low digit, high digit) for up to
-//                     four bit-offset classes, so no register ever has to be shifted.
+//   consumer warps  : two warps share a unit, one 16-row tile each.  Stored words become 8-bit
+//                     mma.m16n8k32 A operands with ONE AND each (no shift: a word holds 8/f
+//                     registers on top of each other, see fq_layout.cuh), the activation digits
+//                     are the B operand, accumulation is exact in s32.  At batch 1 the eight B
+//                     columns carry (low digit, high digit) for up to four bit-offset classes,
+//                     so no register ever has to be shifted.  The loops are compiled once per
+//                     field list (14 variants) and chosen per unit.
+//   output warp     : finishes row pairs (see below) and is the only warp that writes y.
 //   Per group:  y += s * 2^-e * ( sum_fields 2^shift * sum_k field_k * x_int_k  -  z * sum_k x_int_k ).
-// K chunks of one row pair are combined through fp32 partials in a workspace; the last arriver
-// adds them in chunk order, so results do not depend on scheduling.
+// The K chunks of one row pair are computed by different CTAs.  Each unit publishes its row sums
+// as 64-bit words (fp32 value, launch tag) with plain stores; the unit whose chunk index is
+// (row pair mod chunks) hands its own sums to the output warp, which polls the other chunks'
+// words until they carry this launch's tag and adds them in chunk order, so results do not
+// depend on scheduling and no fence or atomic sits on the consumers' path.
 //
 // A whole stack of layers runs as one launch.  Every op's units are dealt to the CTAs in
 // contiguous, K-chunk-major blocks (a CTA needs the activations of one or two chunks only);
@@ -34,7 +40,7 @@ namespace fq {
 #define FQ_CUDA_OK(expr) do { if ((expr) != cudaSuccess) return FQ_ERR_CUDA; } while (0)
 
 #ifndef FQ_GEMV_WARPS
-#define FQ_GEMV_WARPS 16
+#define FQ_GEMV_WARPS 18
 #endif
 #ifndef FQ_GEMV_TPW
 #define FQ_GEMV_TPW 1
