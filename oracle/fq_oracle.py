@@ -194,6 +194,43 @@ def footprint(n_out: Sequence[int], k_in: Sequence[int], bits: Sequence[int]) ->
     return int(_load().fqo_footprint(_p(n), _p(k), _p(b), len(b)))
 
 
+# ---- one-way transitions (Sec. II-C, Sec. III-B) -------------------------------------
+
+def transition(n_out: Sequence[int], k_in: Sequence[int], nested: Sequence[bool], from_bits: Sequence[int],
+               to_bits: Sequence[int]) -> dict:
+    """Memory accounting of moving from one elastic configuration to another, layer by layer.
+
+    The paper asks that a transition only ever lowers a module's bit-width (Sec. III-B, the one-way
+    constraint) and that as little memory as possible has to be brought in (Sec. II-C).  Per layer:
+      nested layer  : the child keeps a prefix of the parent's planes; lowering frees the dropped planes
+                      (N*K*(b0-b1)/8 bytes) and loads nothing, raising loads the re-appended planes;
+                      scale/zero words are shared by every width and never move;
+      packed layer  : widths are separate stored variants; a change frees the old variant and loads the
+                      new one, codes and scale/zero words (4 bytes per group of 128) alike.
+    Returns bytes_freed, bytes_loaded, layers_changed, one_way (no layer goes up) and the footprints of
+    both configurations."""
+    freed = loaded = changed = 0
+    one_way = True
+    for n, k, nest, b0, b1 in zip(n_out, k_in, nested, from_bits, to_bits):
+        n, k, b0, b1 = int(n), int(k), int(b0), int(b1)
+        if b0 == b1:
+            continue
+        changed += 1
+        if b1 > b0:
+            one_way = False
+        if nest:
+            if b1 < b0:
+                freed += n * k * (b0 - b1) // 8
+            else:
+                loaded += n * k * (b1 - b0) // 8
+        else:
+            meta = n * (k // 128) * 4
+            freed += n * k * b0 // 8 + meta
+            loaded += n * k * b1 // 8 + meta
+    return {"bytes_freed": freed, "bytes_loaded": loaded, "layers_changed": changed, "one_way": one_way,
+            "footprint_from": footprint(n_out, k_in, from_bits), "footprint_to": footprint(n_out, k_in, to_bits)}
+
+
 def rel_l2(got: np.ndarray, ref: np.ndarray) -> float:
     """||got - ref||_2 / ||ref||_2 over all elements (0 if both are all-zero)."""
     got = np.asarray(got, np.float64)

@@ -335,3 +335,45 @@ def test_footprint_against_paper_accounting_figures():
     tot_bits = sum(float(v) for v in g["fq_storage_bits"].split())
     gb = 6_476_005_376 * tot_bits / 8 / 1e9
     assert 0.85 * float(g["fq_storage_gb"]) < gb < float(g["fq_storage_gb"])
+
+
+# --------------------------------------------------------------------------- one-way transitions
+
+def test_transition_accounting_closed_forms_and_invariants():
+    import fq_synth as S
+    sh = S.stack_shapes("7b")
+    n, k = [s.n_out for s in sh], [s.k_in for s in sh]
+    g = _golden("paper_accounting.txt")
+    # nested: replacing one attention module (q,k,v,o) of the 8-bit model by its 3-bit version (the
+    # paper's interchangeability example, Sec. III) frees 5 planes of 4 matrices and loads nothing
+    to = [8] * 224
+    to[0:4] = [3] * 4
+    t = O.transition(n, k, [True] * 224, [8] * 224, to)
+    assert t["bytes_freed"] == 4 * 4096 * 4096 * 5 // 8 == 41_943_040 and t["bytes_loaded"] == 0
+    assert t["layers_changed"] == 4 and t["one_way"]
+    # what is freed is exactly the drop in footprint (scale/zero words are shared by all widths)
+    assert t["footprint_from"] - t["footprint_to"] == t["bytes_freed"]
+    assert t["bytes_freed"] / 1e6 < float(g["granularity_mb"])
+    # going back up is not one-way and loads what was freed
+    back = O.transition(n, k, [True] * 224, to, [8] * 224)
+    assert not back["one_way"] and back["bytes_loaded"] == t["bytes_freed"] and back["bytes_freed"] == 0
+    # packed: widths are separate variants, a change swaps codes AND scale/zero words
+    p = O.transition([4096], [4096], [False], [8], [3])
+    meta = 4096 * 32 * 4
+    assert p["bytes_freed"] == 4096 * 4096 + meta and p["bytes_loaded"] == 4096 * 4096 * 3 // 8 + meta and p["one_way"]
+    assert p["bytes_freed"] - p["bytes_loaded"] == p["footprint_from"] - p["footprint_to"]
+    # no change, nothing moves
+    z = O.transition(n, k, [True] * 224, to, to)
+    assert z == {"bytes_freed": 0, "bytes_loaded": 0, "layers_changed": 0, "one_way": True,
+                 "footprint_from": z["footprint_from"], "footprint_to": z["footprint_from"]}
+    # the seeded chains are one-way and every step frees exactly its footprint gap and loads nothing
+    chain = S.config_chain(S.tensor_key(2, 0, S.TENSOR_CHAIN), sh, 12, 7.0, 3.5, 3)
+    for a, b in zip(chain, chain[1:]):
+        t = O.transition(n, k, [True] * 224, a, b)
+        assert t["one_way"] and t["bytes_loaded"] == 0 and t["bytes_freed"] == t["footprint_from"] - t["footprint_to"] > 0
+    # brute force on a tiny mixed case, written out independently
+    nn, kk, nest, f, tt = [32, 64, 16], [256, 128, 384], [True, False, True], [8, 6, 4], [5, 4, 7]
+    t = O.transition(nn, kk, nest, f, tt)
+    assert t["bytes_freed"] == 32 * 256 * 3 // 8 + (64 * 128 * 6 // 8 + 64 * 4)
+    assert t["bytes_loaded"] == (64 * 128 * 4 // 8 + 64 * 4) + 16 * 384 * 3 // 8
+    assert t["layers_changed"] == 3 and not t["one_way"]
