@@ -237,6 +237,7 @@ def config_report(P, device, steps):
         chain = S.config_chain(S.tensor_key(cfg, 0, S.TENSOR_CHAIN), shapes, n_cfg, hi, lo, floor)
         phases = S.stack_phases(shapes)
         rows = []
+        steps_freed, steps_loaded = [], []
         for batch in ((1,) if cfg == 2 else (1, 8)):
             xs = [S.activations(S.tensor_key(cfg, i, S.TENSOR_X), batch, sh.k_in).to(device) for i, sh in enumerate(shapes)]
             ys = [torch.empty((batch, sh.n_out), dtype=torch.float16, device=device) for sh in shapes]
@@ -244,7 +245,12 @@ def config_report(P, device, steps):
             args_free = fq.stack_args(list(range(L)), xs, ys, None)
             for ci, bits in enumerate(chain):
                 t0 = time.perf_counter()
-                fp = fq.fq_set_config([int(b) for b in bits])
+                if ci == 0 or batch != 1:
+                    fp = fq.fq_set_config([int(b) for b in bits])
+                else:                                            # the chain is one-way: every step is a transition
+                    rep = fq.fq_transition([int(b) for b in bits], require_one_way=True)
+                    fp = rep["footprint_to"]
+                    steps_freed.append(rep["bytes_freed"]); steps_loaded.append(rep["bytes_loaded"])
                 switch_us = (time.perf_counter() - t0) * 1e6
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(); fq.fq_gemv_stack_raw(args_dep, batch); e1.record(); torch.cuda.synchronize()
@@ -256,7 +262,11 @@ def config_report(P, device, steps):
                              "ms_per_pass": ms, "GBps": fp / ms / 1e6, "ms_unordered": ms_free, "GBps_unordered": fp / ms_free / 1e6})
             del xs, ys
         entry = {"config": cfg, "workload": f"{model}-shaped stack, nested bit-planes, {n_cfg}-configuration chain",
-                 "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0, "decode": rows}
+                 "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0,
+                 "transitions": {"steps": len(steps_freed), "one_way": True, "bytes_loaded_total": int(sum(steps_loaded)),
+                                 "granularity_bytes_max": int(max(steps_freed)), "granularity_bytes_mean": float(np.mean(steps_freed)),
+                                 "note": "fq_transition per chain step: memory a deployment can release; nothing has to be loaded"},
+                 "decode": rows}
         if cfg == 4:
             bits = chain[-1]
             fq.fq_set_config([int(b) for b in bits])

@@ -47,7 +47,8 @@ enum { FQ_OK = 0,
        FQ_ERR_NOT_PACKED = -6,  /* layer used before fq_pack_layer / fq_set_config          */
        FQ_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, out of memory...) */
        FQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait ran out (see fq_status)       */
-       FQ_ERR_SCRATCH = -9 };   /* problem needs more than the built-in scratch (fq_gemv_static) */
+       FQ_ERR_SCRATCH = -9,     /* problem needs more than the built-in scratch (fq_gemv_static) */
+       FQ_ERR_ONE_WAY = -10 };  /* a layer would go to a higher bit-width (fq_transition)    */
 
 #define FQ_MAX_BATCH 8          /* decode batch handled by the GEMV family */
 
@@ -99,6 +100,27 @@ int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int gro
  * and nothing is enqueued on `stream`. */
 int fq_set_config(fq_ctx* ctx, const uint8_t* bits_host, int n_layers,
                   uint64_t* footprint_bytes_host, void* stream);
+
+/* One-way transition to another elastic configuration (Sec. III-B: a module may only move to a
+ * lower bit-width, which keeps the memory traffic of a transition small; Sec. II-C: what has to be
+ * brought into memory on a switch should be minimal).  Same arguments and checks as fq_set_config;
+ * on success the configuration is active and `report_host` (may be NULL) says what the step costs in
+ * a deployment that keeps only the active variants resident:
+ *   nested (PLANES) layer: lowering frees the dropped planes, N*K*(b0-b1)/8 bytes, and loads nothing;
+ *                          raising loads the re-appended planes; scale/zero words never move.
+ *   PACKED layer         : a change frees the old variant and loads the new one (codes + scale/zero).
+ * The library itself keeps every registered variant resident: nothing is copied or released here.
+ * require_one_way != 0: a configuration that raises any layer returns FQ_ERR_ONE_WAY and changes nothing. */
+typedef struct fq_transition_report {
+    uint64_t bytes_freed;       /* memory a deployment can release after this step               */
+    uint64_t bytes_loaded;      /* memory it has to bring in before this step                    */
+    uint64_t footprint_from;    /* footprint of the configuration that was active                */
+    uint64_t footprint_to;      /* footprint of the new configuration                            */
+    int layers_changed;
+    int one_way;                /* 1: no layer goes to a higher bit-width                        */
+} fq_transition_report;
+int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
+                  fq_transition_report* report_host, void* stream);
 
 /* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.

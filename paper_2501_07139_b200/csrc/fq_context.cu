@@ -131,6 +131,7 @@ const char* fq_strerror(int code)
         case FQ_ERR_CUDA: return "CUDA runtime error";
         case FQ_ERR_TIMEOUT: return "device-side wait timed out";
         case FQ_ERR_SCRATCH: return "layer needs more than the built-in scratch";
+        case FQ_ERR_ONE_WAY: return "transition would raise a layer's bit-width";
         default: return "unknown error";
     }
 }
@@ -245,6 +246,42 @@ int fq_set_config(fq_ctx* ctx, const uint8_t* bits_host, int n_layers, uint64_t*
         if (L.registered) L.active_bits = bits_host[i++];
     ctx->config_epoch++;
     if (footprint_bytes_host) *footprint_bytes_host = total;
+    return FQ_OK;
+}
+
+int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
+                  fq_transition_report* report_host, void* stream)
+{
+    if (!ctx || !to_bits_host) return FQ_ERR_ARG;
+    int registered = 0;
+    for (const Layer& L : ctx->layers) registered += L.registered ? 1 : 0;
+    if (n_layers != registered) return FQ_ERR_ARG;
+    fq_transition_report rep{};
+    rep.one_way = 1;
+    int i = 0;
+    for (const Layer& L : ctx->layers) {
+        if (!L.registered) continue;
+        const int b0 = L.active_bits, b1 = to_bits_host[i++];
+        if (b1 < 2 || b1 > 8) return FQ_ERR_BITS;
+        if (!active_variant(L, b1)) return FQ_ERR_NO_VARIANT;
+        const uint64_t nk = (uint64_t)L.n_out * (uint64_t)L.k_in;
+        const uint64_t meta = (uint64_t)L.n_out * (uint64_t)(L.k_in / kGroup) * 4u;
+        rep.footprint_from += nk * (uint64_t)b0 / 8u + meta;
+        if (b0 == b1) continue;
+        rep.layers_changed++;
+        if (b1 > b0) rep.one_way = 0;
+        if (L.fmt == FQ_FMT_PLANES) {
+            if (b1 < b0) rep.bytes_freed += nk * (uint64_t)(b0 - b1) / 8u;
+            else rep.bytes_loaded += nk * (uint64_t)(b1 - b0) / 8u;
+        } else {
+            rep.bytes_freed += nk * (uint64_t)b0 / 8u + meta;
+            rep.bytes_loaded += nk * (uint64_t)b1 / 8u + meta;
+        }
+    }
+    if (require_one_way && !rep.one_way) return FQ_ERR_ONE_WAY;
+    const int rc = fq_set_config(ctx, to_bits_host, n_layers, &rep.footprint_to, stream);
+    if (rc != FQ_OK) return rc;
+    if (report_host) *report_host = rep;
     return FQ_OK;
 }
 

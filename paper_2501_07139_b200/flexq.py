@@ -22,8 +22,13 @@ _lib = None
 EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
-    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static",
+    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition",
 ]
+
+
+class TransitionReport(C.Structure):
+    _fields_ = [("bytes_freed", C.c_uint64), ("bytes_loaded", C.c_uint64), ("footprint_from", C.c_uint64),
+                ("footprint_to", C.c_uint64), ("layers_changed", C.c_int), ("one_way", C.c_int)]
 
 
 class FlexQError(RuntimeError):
@@ -53,6 +58,7 @@ def lib():
     L.fq_quantize_layer.argtypes = [vp, i, i, i, i, vp, vp, vp, vp]
     L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
     L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
+    L.fq_transition.argtypes = [vp, vp, i, i, C.POINTER(TransitionReport), vp]
     L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
     L.fq_gemv_static.argtypes = [vp, i, vp, vp, vp]
@@ -153,6 +159,15 @@ class FlexQ:
         fp = C.c_uint64(0)
         _check(lib().fq_set_config(self._h, arr, len(bits), C.byref(fp), _stream()), "fq_set_config")
         return int(fp.value)
+
+    def fq_transition(self, bits: Sequence[int], require_one_way: bool = True) -> dict:
+        arr = (C.c_uint8 * len(bits))(*[int(b) for b in bits])
+        rep = TransitionReport()
+        _check(lib().fq_transition(self._h, arr, len(bits), 1 if require_one_way else 0, C.byref(rep), _stream()),
+               "fq_transition")
+        return {"bytes_freed": int(rep.bytes_freed), "bytes_loaded": int(rep.bytes_loaded),
+                "layers_changed": int(rep.layers_changed), "one_way": bool(rep.one_way),
+                "footprint_from": int(rep.footprint_from), "footprint_to": int(rep.footprint_to)}
 
     def fq_storage_bytes(self) -> int:
         return int(lib().fq_storage_bytes(self._h))
