@@ -48,7 +48,8 @@ enum { FQ_OK = 0,
        FQ_ERR_CUDA = -7,        /* a CUDA runtime call failed (no device, out of memory...) */
        FQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait ran out (see fq_status)       */
        FQ_ERR_SCRATCH = -9,     /* problem needs more than the built-in scratch (fq_gemv_static) */
-       FQ_ERR_ONE_WAY = -10 };  /* a layer would go to a higher bit-width (fq_transition)    */
+       FQ_ERR_ONE_WAY = -10,    /* a layer would go to a higher bit-width (fq_transition)    */
+       FQ_ERR_IO = -11 };       /* file could not be opened, read or written, or is malformed */
 
 #define FQ_MAX_BATCH 8          /* decode batch handled by the GEMV family */
 
@@ -121,6 +122,18 @@ typedef struct fq_transition_report {
 } fq_transition_report;
 int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
                   fq_transition_report* report_host, void* stream);
+
+/* The ensemble on disk (Sec. III / V-B: the stored quantized variants whose total size is the paper's
+ * "storage cost").  fq_save writes every registered variant of every layer, exactly as stored on the
+ * device, plus shapes, formats and the active configuration; it synchronises the device.
+ * File (little-endian): "FLEXQ1\0\0", u32 n_layers, u32 0; per layer u32 registered, n_out, k_in, fmt,
+ * active_bits, variant_mask (bit b = a variant of b bits follows); per variant u64 bytes, then the bytes.
+ * fq_load registers the file's layers in `ctx` (created with at least as many layers, none registered yet)
+ * and activates the saved configuration.  Unlike fq_pack_layer it ALLOCATES the device buffers itself
+ * (cudaMalloc); the context owns them until fq_destroy.  Errors: FQ_ERR_ARG (path, context state),
+ * FQ_ERR_IO (open / read / write / malformed file), FQ_ERR_CUDA. */
+int fq_save(fq_ctx* ctx, const char* path, uint64_t* bytes_written_host);
+int fq_load(fq_ctx* ctx, const char* path);
 
 /* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.

@@ -1,5 +1,6 @@
 // C ABI entry points: context, layer registry, configuration / footprint accountant,
 // argument checks and dispatch to the kernels.
+#include <cstdio>
 #include <cstring>
 #include <new>
 
@@ -132,6 +133,7 @@ const char* fq_strerror(int code)
         case FQ_ERR_TIMEOUT: return "device-side wait timed out";
         case FQ_ERR_SCRATCH: return "layer needs more than the built-in scratch";
         case FQ_ERR_ONE_WAY: return "transition would raise a layer's bit-width";
+        case FQ_ERR_IO: return "file could not be opened, read or written, or is malformed";
         default: return "unknown error";
     }
 }
@@ -172,6 +174,7 @@ int fq_destroy(fq_ctx* ctx)
         if (ctx->stack_dev) cudaFree(ctx->stack_dev);
         if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
         if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
+        for (void* p : ctx->owned) cudaFree(p);
     }
     delete ctx;
     return FQ_OK;
@@ -282,6 +285,105 @@ int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int re
     const int rc = fq_set_config(ctx, to_bits_host, n_layers, &rep.footprint_to, stream);
     if (rc != FQ_OK) return rc;
     if (report_host) *report_host = rep;
+    return FQ_OK;
+}
+
+namespace {
+const char kFileMagic[8] = {'F', 'L', 'E', 'X', 'Q', '1', 0, 0};
+constexpr size_t kIoChunk = 32u << 20;            // device <-> file staging, bytes per copy
+struct FileCloser { FILE* f; ~FileCloser() { if (f) std::fclose(f); } };
+size_t variant_store_bytes(const Layer& L, int b) { return (size_t)store_bytes(L.n_out, L.k_in, b); }
+}  // namespace
+
+int fq_save(fq_ctx* ctx, const char* path, uint64_t* bytes_written_host)
+{
+    if (!ctx || !path) return FQ_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    FQ_CUDA_OK(cudaDeviceSynchronize());
+    FileCloser fc{std::fopen(path, "wb")};
+    if (!fc.f) return FQ_ERR_IO;
+    std::vector<char> stage(kIoChunk);
+    uint64_t written = 0;
+    auto put = [&](const void* p, size_t n) { if (std::fwrite(p, 1, n, fc.f) != n) return false; written += n; return true; };
+    const uint32_t head[2] = {(uint32_t)ctx->layers.size(), 0u};
+    if (!put(kFileMagic, 8) || !put(head, 8)) return FQ_ERR_IO;
+    for (const Layer& L : ctx->layers) {
+        uint32_t mask = 0;
+        for (int b = 2; b <= 8; b++) if (L.var[b].present) mask |= 1u << b;
+        const uint32_t rec[6] = {L.registered ? 1u : 0u, (uint32_t)L.n_out, (uint32_t)L.k_in, (uint32_t)L.fmt,
+                                 (uint32_t)L.active_bits, mask};
+        if (!put(rec, sizeof rec)) return FQ_ERR_IO;
+        for (int b = 2; b <= 8; b++) {
+            if (!L.var[b].present) continue;
+            const uint64_t bytes = variant_store_bytes(L, b);
+            if (!put(&bytes, 8)) return FQ_ERR_IO;
+            for (uint64_t off = 0; off < bytes; off += kIoChunk) {
+                const size_t n = (size_t)(bytes - off < kIoChunk ? bytes - off : kIoChunk);
+                FQ_CUDA_OK(cudaMemcpy(stage.data(), static_cast<const char*>(L.var[b].store) + off, n, cudaMemcpyDeviceToHost));
+                if (!put(stage.data(), n)) return FQ_ERR_IO;
+            }
+        }
+    }
+    if (std::fflush(fc.f) != 0) return FQ_ERR_IO;
+    if (bytes_written_host) *bytes_written_host = written;
+    return FQ_OK;
+}
+
+int fq_load(fq_ctx* ctx, const char* path)
+{
+    if (!ctx || !path) return FQ_ERR_ARG;
+    for (const Layer& L : ctx->layers) if (L.registered) return FQ_ERR_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    FileCloser fc{std::fopen(path, "rb")};
+    if (!fc.f) return FQ_ERR_IO;
+    auto get = [&](void* p, size_t n) { return std::fread(p, 1, n, fc.f) == n; };
+    char magic[8];
+    uint32_t head[2];
+    if (!get(magic, 8) || std::memcmp(magic, kFileMagic, 8) != 0 || !get(head, 8)) return FQ_ERR_IO;
+    if (head[0] > ctx->layers.size()) return FQ_ERR_ARG;
+    std::vector<char> stage(kIoChunk);
+    std::vector<Layer> loaded(head[0]);
+    std::vector<void*> bufs;
+    int rc = FQ_OK;
+    for (uint32_t i = 0; i < head[0] && rc == FQ_OK; i++) {
+        uint32_t rec[6];
+        if (!get(rec, sizeof rec)) { rc = FQ_ERR_IO; break; }
+        Layer& L = loaded[i];
+        L.registered = rec[0] != 0;
+        L.n_out = (int)rec[1]; L.k_in = (int)rec[2]; L.fmt = (int)rec[3]; L.active_bits = (int)rec[4];
+        if (!L.registered) { if (rec[5] != 0) rc = FQ_ERR_IO; continue; }
+        const bool planes = L.fmt == FQ_FMT_PLANES;
+        const uint32_t mask = rec[5];
+        const bool shape_ok = (L.fmt == FQ_FMT_PACKED || planes) && L.n_out >= 1 && L.k_in >= 1 && L.k_in % kGroup == 0;
+        const bool mask_ok = mask != 0 && (mask & ~0x1FCu) == 0 && (!planes || mask == (1u << 8));
+        const bool active_ok = L.active_bits >= 2 && L.active_bits <= 8 && (planes || (mask & (1u << L.active_bits)));
+        if (!shape_ok || !mask_ok || !active_ok) { rc = FQ_ERR_IO; break; }
+        for (int b = 2; b <= 8 && rc == FQ_OK; b++) {
+            if (!(rec[5] & (1u << b))) continue;
+            uint64_t bytes = 0;
+            if (!get(&bytes, 8) || bytes != variant_store_bytes(L, b)) { rc = FQ_ERR_IO; break; }
+            void* dev = nullptr;
+            if (cudaMalloc(&dev, (size_t)bytes) != cudaSuccess) { rc = FQ_ERR_CUDA; break; }
+            bufs.push_back(dev);
+            for (uint64_t off = 0; off < bytes && rc == FQ_OK; off += kIoChunk) {
+                const size_t n = (size_t)(bytes - off < kIoChunk ? bytes - off : kIoChunk);
+                if (!get(stage.data(), n)) rc = FQ_ERR_IO;
+                else if (cudaMemcpy(static_cast<char*>(dev) + off, stage.data(), n, cudaMemcpyHostToDevice) != cudaSuccess) rc = FQ_ERR_CUDA;
+            }
+            L.var[b].present = true;
+            L.var[b].store = dev;
+        }
+    }
+    if (rc != FQ_OK) {                                   // a failing call changes nothing
+        for (void* p : bufs) cudaFree(p);
+        return rc;
+    }
+    for (uint32_t i = 0; i < head[0]; i++) ctx->layers[i] = loaded[i];
+    ctx->owned.insert(ctx->owned.end(), bufs.begin(), bufs.end());
+    ctx->config_epoch++;
+    ctx->stack_valid = false;
     return FQ_OK;
 }
 

@@ -74,6 +74,7 @@ struct Ctx {
     // prefill: dequantised bf16 copy of the layer being multiplied
     char* gemm_ws = nullptr;
     size_t gemm_ws_bytes = 0;
+    std::vector<void*> owned;    // device buffers allocated by fq_load, freed by fq_destroy
     uint64_t config_epoch = 0;
     unsigned launch_epoch = 0;   // tag of the split-K partials of the latest decode launch (never 0)
     uint64_t stack_key = 0;      // hash of the op list that is currently uploaded

@@ -22,7 +22,7 @@ _lib = None
 EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
-    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition",
+    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load",
 ]
 
 
@@ -59,6 +59,8 @@ def lib():
     L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
     L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
     L.fq_transition.argtypes = [vp, vp, i, i, C.POINTER(TransitionReport), vp]
+    L.fq_save.argtypes = [vp, C.c_char_p, C.POINTER(u64)]
+    L.fq_load.argtypes = [vp, C.c_char_p]
     L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
     L.fq_gemv_static.argtypes = [vp, i, vp, vp, vp]
@@ -168,6 +170,16 @@ class FlexQ:
         return {"bytes_freed": int(rep.bytes_freed), "bytes_loaded": int(rep.bytes_loaded),
                 "layers_changed": int(rep.layers_changed), "one_way": bool(rep.one_way),
                 "footprint_from": int(rep.footprint_from), "footprint_to": int(rep.footprint_to)}
+
+    def fq_save(self, path: str) -> int:
+        """Writes every stored variant to `path`; returns the bytes written."""
+        n = C.c_uint64(0)
+        _check(lib().fq_save(self._h, os.fsencode(path), C.byref(n)), "fq_save")
+        return int(n.value)
+
+    def fq_load(self, path: str):
+        """Registers the layers of a file written by fq_save (the library allocates their device buffers)."""
+        _check(lib().fq_load(self._h, os.fsencode(path)), "fq_load")
 
     def fq_storage_bytes(self) -> int:
         return int(lib().fq_storage_bytes(self._h))
