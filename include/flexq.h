@@ -135,6 +135,33 @@ int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int re
 int fq_save(fq_ctx* ctx, const char* path, uint64_t* bytes_written_host);
 int fq_load(fq_ctx* ctx, const char* path);
 
+/* Tree search for an ensemble of elastic configurations (Sec. III-B, Algorithm 1), on tables instead of
+ * perplexity runs.  n_modules modules, n_levels stored precisions ordered from n_up (level 0) down to n_low
+ * (level n_levels-1); a configuration is one level per module.  Host tables, all [n_modules][n_levels]:
+ *   cost : what calibrationEval adds when module m sits at level l (cost[m][0] = 0); a configuration is
+ *          evaluated as the sum over its modules;
+ *   sens : the pre-generated sensitivity of replacing module m of QM(n_up) by level l (smaller = ranked higher);
+ *   foot : bytes of module m stored at level l.
+ * Each iteration generates, for the last configuration of each of the (at most) `stems` ensembles, every
+ * successor that lowers ONE module by ONE level (the one-way rule), keeps the `branches` least sensitive per
+ * ensemble, evaluates them, ranks by (cost, footprint, generation order) and keeps the best `stems` distinct
+ * ones.  It ends when every module is at n_low, after n_modules*(n_levels-1) steps, and returns the ensemble
+ * with the smallest sum of cost over its configurations.
+ *   chain_out uint8 [n_modules*(n_levels-1)+1][n_modules]: level per module, first row all 0.  Host memory. */
+int fq_search_chain(const double* cost, const double* sens, const uint64_t* foot, int n_modules, int n_levels,
+                    int stems, int branches, uint8_t* chain_out, int* n_states_out, double* curve_cost_out);
+
+/* Pruning of mid-precision modules (Sec. III-C).  Every (module, mid level) pair is ranked by how many
+ * configurations of `chain` use it, ties by use at lower footprints (later in the chain); the lowest-ranked
+ * floor(fraction * pairs) are dropped.  A configuration that used a dropped pair falls to the next lower stored
+ * level.  dropped_out uint8 [n_modules][n_levels] flags; storage = sum of foot over the kept pairs. */
+int fq_prune_chain(const uint8_t* chain, int n_states, int n_modules, int n_levels, const uint64_t* foot, double fraction,
+                   uint8_t* pruned_chain_out, uint8_t* dropped_out, uint64_t* storage_before_out, uint64_t* storage_after_out);
+
+/* Output error of a layer, the stand-in for the calibration-set evaluation (Sec. III-B): writes
+ * sums_dev[0] = sum (a-b)^2 and sums_dev[1] = sum b^2 over n bf16 values (device pointers). */
+int fq_sqdiff(const uint16_t* a_bf16_dev, const uint16_t* b_bf16_dev, size_t n, double* sums_dev, void* stream);
+
 /* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.
  * Enqueues kernels on `stream`; does not synchronise. */

@@ -22,7 +22,7 @@ _lib = None
 EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
-    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load",
+    "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load", "fq_search_chain", "fq_prune_chain", "fq_sqdiff",
 ]
 
 
@@ -61,6 +61,9 @@ def lib():
     L.fq_transition.argtypes = [vp, vp, i, i, C.POINTER(TransitionReport), vp]
     L.fq_save.argtypes = [vp, C.c_char_p, C.POINTER(u64)]
     L.fq_load.argtypes = [vp, C.c_char_p]
+    L.fq_search_chain.argtypes = [vp, vp, vp, i, i, i, i, vp, C.POINTER(i), C.POINTER(C.c_double)]
+    L.fq_prune_chain.argtypes = [vp, i, i, i, vp, C.c_double, vp, vp, C.POINTER(u64), C.POINTER(u64)]
+    L.fq_sqdiff.argtypes = [vp, vp, C.c_size_t, vp, vp]
     L.fq_gemv.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_batched.argtypes = [vp, i, vp, i, vp, vp]
     L.fq_gemv_static.argtypes = [vp, i, vp, vp, vp]
@@ -98,6 +101,43 @@ def _check(rc: int, where: str) -> int:
     if rc != 0:
         raise FlexQError(rc, where)
     return rc
+
+
+def fq_search_chain(cost, sens, foot, stems: int, branches: int):
+    """Algorithm 1 on host tables [module][level]; returns (chain as a list of level lists, curve cost)."""
+    import numpy as np
+    c = np.ascontiguousarray(cost, np.float64)
+    s_ = np.ascontiguousarray(sens, np.float64)
+    f = np.ascontiguousarray(foot, np.uint64)
+    m, lv = c.shape
+    chain = np.zeros((m * (lv - 1) + 1, m), np.uint8)
+    n_states, curve = C.c_int(0), C.c_double(0.0)
+    _check(lib().fq_search_chain(c.ctypes.data, s_.ctypes.data, f.ctypes.data, m, lv, stems, branches, chain.ctypes.data,
+                                 C.byref(n_states), C.byref(curve)), "fq_search_chain")
+    return chain[:n_states.value].tolist(), float(curve.value)
+
+
+def fq_prune_chain(chain, n_levels: int, foot, fraction: float):
+    """Sec. III-C; returns (pruned chain, set of dropped (module, level), storage before, storage after)."""
+    import numpy as np
+    ch = np.ascontiguousarray(chain, np.uint8)
+    f = np.ascontiguousarray(foot, np.uint64)
+    n_states, m = ch.shape
+    out = np.zeros_like(ch)
+    dropped = np.zeros((m, n_levels), np.uint8)
+    before, after = C.c_uint64(0), C.c_uint64(0)
+    _check(lib().fq_prune_chain(ch.ctypes.data, n_states, m, n_levels, f.ctypes.data, float(fraction), out.ctypes.data,
+                                dropped.ctypes.data, C.byref(before), C.byref(after)), "fq_prune_chain")
+    return out.tolist(), {(int(a), int(b)) for a, b in zip(*np.nonzero(dropped))}, int(before.value), int(after.value)
+
+
+def fq_sqdiff(a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    """Device tensor [sum (a-b)^2, sum b^2] (float64) over two bf16 tensors of the same size."""
+    assert a.dtype == torch.bfloat16 and b.dtype == torch.bfloat16 and a.is_contiguous() and b.is_contiguous()
+    assert a.numel() == b.numel()
+    out = torch.empty(2, dtype=torch.float64, device=a.device)
+    _check(lib().fq_sqdiff(a.data_ptr(), b.data_ptr(), a.numel(), out.data_ptr(), _stream()), "fq_sqdiff")
+    return out
 
 
 def fq_quantize_layer(w: torch.Tensor, bits: int, group: int = 128):
