@@ -267,6 +267,34 @@ def config_report(P, device, steps):
                                  "granularity_bytes_max": int(max(steps_freed)), "granularity_bytes_mean": float(np.mean(steps_freed)),
                                  "note": "fq_transition per chain step: memory a deployment can release; nothing has to be loaded"},
                  "decode": rows}
+        if cfg == 2:
+            # the offline side on the same stack: tables measured with the prefill kernel, tree search, pruning
+            from paper_2501_07139_b200 import search as SR
+            levels = [8, 5, 3]
+            mods = {}
+            for i, sh in enumerate(shapes):
+                mods.setdefault((sh.block, sh.module), []).append(i)
+            modules = [mods[k] for k in sorted(mods)]
+            calib = {kk: S.activations(S.tensor_key(cfg, kk, S.TENSOR_X), 2048, kk, torch.bfloat16, device=device)
+                     for kk in sorted({sh.k_in for sh in shapes})}
+            torch.cuda.synchronize(); t0 = time.perf_counter()
+            cost, sens, foot = SR.module_tables(fq, shapes, modules, levels, calib, 256)
+            t_tab = time.perf_counter() - t0
+            t0 = time.perf_counter()
+            ens, curve = P.fq_search_chain(cost, sens, foot, 2, 3)
+            t_search = time.perf_counter() - t0
+            pruned, dropped, before, after = P.fq_prune_chain(ens, len(levels), foot, 0.5)
+            fps = [sum(foot[m][l] for m, l in enumerate(st)) for st in ens]
+            entry["ensemble_search"] = {
+                "modules": len(modules), "levels_bits": levels, "stems": 2, "branches": 3, "calibration_tokens": 2048,
+                "evaluation": "relative output error of the linear layers (stand-in for calibration perplexity)",
+                "table_seconds_gpu": t_tab, "table_fq_gemm_calls": len(shapes) * len(levels), "search_seconds_host": t_search,
+                "configurations": len(ens), "curve_cost": curve,
+                "granularity_bytes_max": int(max(a - b for a, b in zip(fps, fps[1:]))),
+                "code_bytes_first_last": [int(fps[0]), int(fps[-1])],
+                "pruning_50pct": {"dropped_mid_modules": len(dropped), "storage_code_bytes_before": before,
+                                  "storage_code_bytes_after": after}}
+            del calib
         if cfg == 4:
             bits = chain[-1]
             fq.fq_set_config([int(b) for b in bits])
