@@ -277,3 +277,34 @@ def test_stack_after_single_calls_with_split_k(P):
     ref = O.gemv(*layers[1], 3, bits_of(xs[1]))
     assert O.rel_l2(f64_of(y_single[1]), ref) <= GEMV_TOL
     fq.fq_destroy()
+
+
+def test_gemv_stack_phases_carry_real_data_dependencies(P):
+    """A chain in which every op reads what the previous phase wrote (x of op i+1 IS y of op i): the values
+    must equal those of separate calls in sequence, launch after launch.  A phase that started before the
+    previous one had published all of its outputs would read stale or poisoned activations."""
+    dims = [1024, 2048, 1024, 4096, 1024]                      # k_in of op 0, then n_out of every op
+    bits = [8, 4, 3, 5]
+    L = len(bits)
+    fq = P.FlexQ(L)
+    for i in range(L):
+        fq.fq_pack_layer(i, *to_dev(*make_layer(101, i, dims[i + 1], dims[i], bits[i])), bits[i], P.FQ_FMT_PACKED)
+    x0 = (x_fp16(101, 0, 1, dims[0]) * 4).cuda()
+    # reference: one call after the other; scale so that the chain neither dies out nor overflows
+    seq = [x0[0]]
+    for i in range(L):
+        y = torch.empty(dims[i + 1], dtype=torch.float16, device="cuda")
+        fq.fq_gemv(i, seq[-1], y)
+        seq.append(y)
+    torch.cuda.synchronize()
+    assert all(torch.isfinite(t).all() and t.abs().max() > 0 for t in seq)
+    bufs = [x0[0].clone()] + [torch.empty(dims[i + 1], dtype=torch.float16, device="cuda") for i in range(L)]
+    for rep in range(25):
+        for t in bufs[1:]:
+            t.fill_(float("nan"))                              # poison: an early reader would see NaN
+        fq.fq_gemv_stack(list(range(L)), bufs[:-1], bufs[1:], list(range(L)), 1)
+        torch.cuda.synchronize()
+        for i in range(L):
+            assert torch.equal(bufs[i + 1], seq[i + 1]), (rep, i)
+    assert fq.fq_status() == 0
+    fq.fq_destroy()
