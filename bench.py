@@ -319,23 +319,38 @@ def config_report(P, device, steps):
     return out
 
 
-def oracle_sample(shapes, bits, n_layers, device_for_gen):
-    """Times the CPU oracle's GEMV on the first `n_layers` matrices of the workload.
-    Returns (bytes processed, seconds, description)."""
+def oracle_inputs(shapes, bits, n_layers, device_for_gen):
+    """Quantised matrices and activations of the first `n_layers` matrices of the workload, as the CPU oracle takes them."""
     from oracle import fq_oracle as O
     O.build()
-    total_bytes, total_s = 0, 0.0
+    items = []
     for i in range(n_layers):
         sh, b = shapes[i], int(bits[i])
         w = S.weight_rows(S.tensor_key(CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device_for_gen)
         codes, sc, zr = O.quantize(w.cpu().numpy(), b)
         x = S.activations(S.tensor_key(CONFIG_ID, i, S.TENSOR_X), 1, sh.k_in, torch.float16)
         xb = x.view(torch.int16).numpy().view(np.uint16)
+        items.append((codes, sc, zr, b, xb, sh.n_out * sh.k_in * b // 8 + sh.n_out * (sh.k_in // 128) * 4))
+    return items
+
+
+def oracle_pass(items):
+    """One timed pass of the CPU oracle's GEMV over `items`.  Returns (bytes processed, seconds)."""
+    from oracle import fq_oracle as O
+    total_bytes, total_s = 0, 0.0
+    for codes, sc, zr, b, xb, nbytes in items:
         t0 = time.perf_counter()
         O.gemv(codes, sc, zr, b, xb)
         total_s += time.perf_counter() - t0
-        total_bytes += sh.n_out * sh.k_in * b // 8 + sh.n_out * (sh.k_in // 128) * 4
-    return total_bytes, total_s, f"oracle GEMV over the first {n_layers} matrices (block 0) of the stack, single thread"
+        total_bytes += nbytes
+    return total_bytes, total_s
+
+
+def oracle_desc(n_layers):
+    return f"oracle GEMV over the first {n_layers} matrices of the stack ({n_layers / 7:.2g} blocks), single thread"
+
+
+REF_BUDGET_S = 150.0          # CPU seconds the whole reference run may take, over all its steps
 
 
 def run_reference(args, rank):
@@ -344,10 +359,20 @@ def run_reference(args, rank):
     shapes = S.stack_shapes("7b", args.blocks)
     bits = S.draw_bits(S.tensor_key(CONFIG_ID, 0, S.TENSOR_BITS), len(shapes), BIT_CHOICES)
     gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
-    n_layers = min(args.ref_layers, len(shapes))
+    items = oracle_inputs(shapes, bits, min(args.ref_layers, len(shapes)), gen_dev)
+    # bound the run: one untimed pass gives each matrix's cost, a step is the longest prefix of the sample
+    # that keeps (warmup + steps) passes inside the budget
+    per = [oracle_pass([it])[1] for it in items]
+    n_layers, acc = 0, 0.0
+    for t in per:
+        if n_layers >= 1 and (acc + t) * (args.warmup + args.steps) > REF_BUDGET_S:
+            break
+        acc += t; n_layers += 1
+    items = items[:n_layers]
+    desc = oracle_desc(n_layers)
     times, byts = [], 0
     for step in range(args.warmup + args.steps):
-        byts, secs, desc = oracle_sample(shapes, bits, n_layers, gen_dev)
+        byts, secs = oracle_pass(items)
         if step >= args.warmup:
             times.append(secs)
     t = float(np.mean(times))
@@ -372,7 +397,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--blocks", type=int, default=32, help="decoder blocks of the 7B-shaped stack (32 = full)")
-    ap.add_argument("--ref-layers", type=int, default=7, help="matrices the CPU oracle is timed on")
+    ap.add_argument("--ref-layers", type=int, default=7,
+                    help="--impl reference: matrices per step at most (fewer when warmup + steps would pass the time budget)")
+    ap.add_argument("--cpu-layers", type=int, default=14, help="matrices the cpu_baseline leg times the CPU oracle on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill (tensor-core GEMM) leg")
     ap.add_argument("--prefill-steps", type=int, default=3)
@@ -526,9 +553,10 @@ def main():
                          "kernel": "gemm_kernel (tcgen05) + dequant_kernel; flops = 2*M*N*K per matrix"},
         }
     if not args.no_cpu_baseline:
-        n_layers = min(args.ref_layers, L)
-        byts, secs, desc = oracle_sample(shapes, bits, n_layers, device)
-        line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
+        n_layers = min(args.cpu_layers, L)
+        byts, secs = oracle_pass(oracle_inputs(shapes, bits, n_layers, device))
+        line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": oracle_desc(n_layers)}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
