@@ -78,21 +78,28 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
     op.n_units = op.n_chunks * op.n_rp;
     if ((long long)op.n_chunks * op.n_rp * 1024 >= (1ll << 31)) return FQ_ERR_SHAPE;   // 32-bit unit arithmetic on the device
+    if (batch == 1 && L.k_in > gemv1_max_k()) return FQ_ERR_SHAPE;                   // a strip's activations stay in shared memory
     op.phase = -1;
     op.rot = 0;
     return FQ_OK;
 }
 
+// Split-K scratch of one op.  Batch 1: one tagged word per (strip, blob, row) -- only strips that two CTAs
+// share are ever written.  Batch 2..8: one tagged word per (row pair, K chunk, row, batch entry).
 size_t op_partial_bytes(const GemvOp& op, int max_batch)
 {
     if (op.n_chunks <= 1) return 0;
+    if (max_batch <= 1) return (size_t)op.n_rp * op.n_kb * 32 * sizeof(unsigned long long);
     return (size_t)op.n_rp * op.n_chunks * gemv_partial_bytes_per_unit(max_batch);
 }
 
-uint64_t hash_mix(uint64_t h, uint64_t v)
+// Scratch that a registered layer can need in one launch, whatever its active variant and the batch.
+size_t layer_partial_bytes(int n_out, int k_in)
 {
-    h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2);
-    return h;
+    const size_t n_rp = (size_t)row_pairs(n_out), n_kb = (size_t)k_blobs(k_in);
+    const size_t b1 = n_rp * n_kb * 32 * sizeof(unsigned long long);
+    const size_t b8 = n_rp * n_kb * gemv_partial_bytes_per_unit(FQ_MAX_BATCH);     // chunks are whole blobs
+    return (size_t)round_up((int64_t)(b1 > b8 ? b1 : b8), 256);
 }
 
 }  // namespace
@@ -102,7 +109,7 @@ namespace fq {
 int ensure_workspace(Ctx* ctx, size_t bytes)
 {
     if (bytes <= ctx->ws_bytes) return FQ_OK;
-    const size_t want = (size_t)round_up((int64_t)(bytes + bytes / 4), 1 << 20);
+    const size_t want = (size_t)round_up((int64_t)(bytes + bytes / 2), 1 << 20);
     char* p = nullptr;
     FQ_CUDA_OK(cudaDeviceSynchronize());
     FQ_CUDA_OK(cudaMalloc(&p, want));
@@ -172,7 +179,10 @@ int fq_destroy(fq_ctx* ctx)
         if (ctx->ws) cudaFree(ctx->ws);
         if (ctx->status_dev) cudaFree(ctx->status_dev);
         if (ctx->stack_dev) cudaFree(ctx->stack_dev);
-        if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
+        for (int i = 0; i < 2; i++) {
+            if (ctx->stage_host[i]) cudaFreeHost(ctx->stage_host[i]);
+            if (ctx->stage_done[i]) cudaEventDestroy(ctx->stage_done[i]);
+        }
         if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
         for (void* p : ctx->owned) cudaFree(p);
     }
@@ -217,12 +227,20 @@ int fq_pack_layer(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, int gro
     const int rc = launch_pack(codes_dev, scales_dev, zeros_dev, n_out, k_in, bits, fl, store_out_dev,
                                (cudaStream_t)stream);
     if (rc != FQ_OK) return rc;
+    const bool first_variant = !L.registered;
     L.registered = true;
     L.n_out = n_out; L.k_in = k_in; L.fmt = fmt;
     Variant& v = L.var[bits];
     v.present = true; v.store = store_out_dev;
     if (L.active_bits == 0) L.active_bits = bits;
     ctx->config_epoch++;
+    // the decode calls never allocate as long as a launch uses every layer at most once: the scratch for
+    // that is sized here
+    if (first_variant) {
+        ctx->ws_reserved += layer_partial_bytes(n_out, k_in);
+        const int rc2 = ensure_workspace(ctx, kPartialBase + ctx->ws_reserved + 256);
+        if (rc2 != FQ_OK) return rc2;
+    }
     return FQ_OK;
 }
 
@@ -437,7 +455,7 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
     rc = ensure_workspace(ctx, kPartialBase + pb + 256);
     if (rc != FQ_OK) return rc;
     op.partial = reinterpret_cast<unsigned long long*>(ctx->ws + kPartialBase);
-    return launch_gemv_single(ctx, op, (cudaStream_t)stream);
+    return batch == 1 ? launch_gemv1_single(ctx, op, (cudaStream_t)stream) : launch_gemv_single(ctx, op, (cudaStream_t)stream);
 }
 
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream)
@@ -467,38 +485,45 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         for (int i = 1; i < n_ops; i++)
             if (phases_host[i] < phases_host[i - 1] || phases_host[i] > phases_host[i - 1] + 1) return FQ_ERR_ARG;
         n_phases = phases_host[n_ops - 1] + 1;
-        if (n_phases > kMaxPhases) return FQ_ERR_SHAPE;
+        if (n_phases > (batch == 1 ? gemv1_max_phases() : kMaxPhases)) return FQ_ERR_SHAPE;
     }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
+    const cudaStream_t st = (cudaStream_t)stream;
 
-    // The op table only depends on the arguments and the active configuration: reuse the
-    // uploaded copy when neither changed.
-    uint64_t key = hash_mix(0x51ed27, (uint64_t)n_ops);
-    key = hash_mix(key, ctx->config_epoch);
-    key = hash_mix(key, (uint64_t)batch);
+    // The op table only depends on the arguments and the active configuration: the uploaded copy is
+    // reused when every argument word is the same as in the call that built it.
+    std::vector<uint64_t> sig;
+    sig.reserve(4 + 4 * (size_t)n_ops);
+    sig.push_back((uint64_t)n_ops); sig.push_back(ctx->config_epoch); sig.push_back((uint64_t)batch);
+    sig.push_back(phases_host ? 1u : 0u);
     for (int i = 0; i < n_ops; i++) {
-        key = hash_mix(key, (uint64_t)layers_host[i]);
-        key = hash_mix(key, (uint64_t)reinterpret_cast<uintptr_t>(x_dev_host[i]));
-        key = hash_mix(key, (uint64_t)reinterpret_cast<uintptr_t>(y_dev_host[i]));
-        key = hash_mix(key, phases_host ? (uint64_t)phases_host[i] : ~0ull);
+        sig.push_back((uint64_t)(int64_t)layers_host[i]);
+        sig.push_back((uint64_t)reinterpret_cast<uintptr_t>(x_dev_host[i]));
+        sig.push_back((uint64_t)reinterpret_cast<uintptr_t>(y_dev_host[i]));
+        sig.push_back(phases_host ? (uint64_t)(int64_t)phases_host[i] : 0u);
     }
-    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) + (size_t)(n_phases > 0 ? n_phases : 1) * sizeof(long long) +
-                               (size_t)ctx->sm_count * sizeof(int);
-    const size_t hdr_off = (size_t)round_up((int64_t)table_bytes, 16);
-    StackHeader hdr{};
+    const int np = n_phases > 0 ? n_phases : 1;
+    // batch 1:    [GemvOp x n_ops][int phase_total x np]
+    // batch 2..8: [GemvOp x n_ops][long long phase_total x np][int cta_units x sm_count]
+    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) +
+                               (batch == 1 ? (size_t)np * sizeof(int)
+                                           : (size_t)np * sizeof(long long) + (size_t)ctx->sm_count * sizeof(int));
 
-    if (!(ctx->stack_valid && ctx->stack_key == key)) {
-        if (ctx->stack_host_bytes < hdr_off + sizeof(StackHeader)) {
-            if (ctx->stack_host) cudaFreeHost(ctx->stack_host);
-            ctx->stack_host = nullptr; ctx->stack_host_bytes = 0;
-            const size_t want = 2 * (hdr_off + sizeof(StackHeader));
-            FQ_CUDA_OK(cudaMallocHost(&ctx->stack_host, want));
-            ctx->stack_host_bytes = want;
+    if (!(ctx->stack_valid && ctx->stack_sig == sig)) {
+        ctx->stack_valid = false;                           // until the new table is complete
+        // staging buffer: the two take turns; wait for the upload that last read this one
+        const int sb = ctx->stage_next;
+        if (ctx->stage_done[sb]) FQ_CUDA_OK(cudaEventSynchronize(ctx->stage_done[sb]));
+        else FQ_CUDA_OK(cudaEventCreateWithFlags(&ctx->stage_done[sb], cudaEventDisableTiming));
+        if (ctx->stage_host_bytes[sb] < table_bytes) {
+            if (ctx->stage_host[sb]) cudaFreeHost(ctx->stage_host[sb]);
+            ctx->stage_host[sb] = nullptr; ctx->stage_host_bytes[sb] = 0;
+            FQ_CUDA_OK(cudaMallocHost(&ctx->stage_host[sb], 2 * table_bytes));
+            ctx->stage_host_bytes[sb] = 2 * table_bytes;
         }
-        GemvOp* ops = reinterpret_cast<GemvOp*>(ctx->stack_host);
-        long long* phase_total = reinterpret_cast<long long*>(ctx->stack_host + (size_t)n_ops * sizeof(GemvOp));
-        for (int p = 0; p < (n_phases > 0 ? n_phases : 1); p++) phase_total[p] = 0;
+        char* host = ctx->stage_host[sb];
+        GemvOp* ops = reinterpret_cast<GemvOp*>(host);
         size_t ws_need = kPartialBase;
         long long unit_base = 0;
         std::vector<long long> bases(n_ops);
@@ -507,30 +532,47 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             if (rc != FQ_OK) return rc;
             ops[i].phase = phases_host ? phases_host[i] : -1;
             bases[i] = unit_base;
-            unit_base += (long long)ops[i].n_rp * ops[i].n_chunks;
-            if (phases_host) phase_total[phases_host[i]] += ops[i].n_rp;     // one finished row pair = one count
+            unit_base += ops[i].n_units;
             ws_need += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
-        int rc = ensure_workspace(ctx, ws_need + 256);
+        const int rc = ensure_workspace(ctx, ws_need + 256);   // (no allocation when every layer appears once)
         if (rc != FQ_OK) return rc;
         size_t poff = kPartialBase;
         for (int i = 0; i < n_ops; i++) {
             ops[i].partial = reinterpret_cast<unsigned long long*>(ctx->ws + poff);
             poff += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
         }
-        // how many units each CTA of the persistent grid will see (the consumers' loop bound)
-        int* cta_units = reinterpret_cast<int*>(phase_total + (n_phases > 0 ? n_phases : 1));
         const int grid = (int)(unit_base < ctx->sm_count ? unit_base : ctx->sm_count);
         for (int i = 0; i < n_ops; i++) ops[i].rot = (int)(bases[i] % (grid > 0 ? grid : 1));
-        for (int c = 0; c < ctx->sm_count; c++) cta_units[c] = 0;
-        for (int i = 0; i < n_ops; i++)
-            for (int c = 0; c < grid; c++) {
-                int lo, hi;
-                gemv_cta_range(ops[i].n_units, ops[i].rot, c, grid, lo, hi);
-                cta_units[c] += hi - lo;
+        if (batch == 1) {
+            // per phase: CTAs that finish at least one strip (each reports once when its strips are done)
+            int* phase_total = reinterpret_cast<int*>(host + (size_t)n_ops * sizeof(GemvOp));
+            for (int p = 0; p < np; p++) phase_total[p] = 0;
+            if (phases_host) {
+                std::vector<int> last_phase(grid, -1);
+                for (int i = 0; i < n_ops; i++)
+                    for (int c = 0; c < grid; c++)
+                        if (cta_work(ops[i].n_units, ops[i].n_chunks, ops[i].rot, c, grid).finishing(ops[i].n_chunks) > 0 &&
+                            last_phase[c] != phases_host[i]) {
+                            last_phase[c] = phases_host[i];
+                            phase_total[phases_host[i]]++;
+                        }
             }
-        hdr.n_ops = n_ops; hdr.n_phases = n_phases; hdr.total_units = unit_base;
-        std::memcpy(ctx->stack_host + hdr_off, &hdr, sizeof hdr);
+        } else {
+            long long* phase_total = reinterpret_cast<long long*>(host + (size_t)n_ops * sizeof(GemvOp));
+            for (int p = 0; p < np; p++) phase_total[p] = 0;
+            if (phases_host)
+                for (int i = 0; i < n_ops; i++) phase_total[phases_host[i]] += ops[i].n_rp;   // one finished row pair = one count
+            // how many units each CTA of the persistent grid will see (the consumers' loop bound)
+            int* cta_units = reinterpret_cast<int*>(phase_total + np);
+            for (int c = 0; c < ctx->sm_count; c++) cta_units[c] = 0;
+            for (int i = 0; i < n_ops; i++)
+                for (int c = 0; c < grid; c++) {
+                    int lo, hi;
+                    gemv_cta_range(ops[i].n_units, ops[i].rot, c, grid, lo, hi);
+                    cta_units[c] += hi - lo;
+                }
+        }
         if (ctx->stack_dev_bytes < table_bytes) {
             FQ_CUDA_OK(cudaDeviceSynchronize());
             if (ctx->stack_dev) cudaFree(ctx->stack_dev);
@@ -538,14 +580,15 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             FQ_CUDA_OK(cudaMalloc(&ctx->stack_dev, 2 * table_bytes));
             ctx->stack_dev_bytes = 2 * table_bytes;
         }
-        FQ_CUDA_OK(cudaMemcpyAsync(ctx->stack_dev, ctx->stack_host, table_bytes, cudaMemcpyHostToDevice,
-                                   (cudaStream_t)stream));
-        ctx->stack_key = key;
+        FQ_CUDA_OK(cudaMemcpyAsync(ctx->stack_dev, host, table_bytes, cudaMemcpyHostToDevice, st));
+        FQ_CUDA_OK(cudaEventRecord(ctx->stage_done[sb], st));
+        ctx->stage_next = sb ^ 1;
+        ctx->stack_hdr.n_ops = n_ops; ctx->stack_hdr.n_phases = n_phases; ctx->stack_hdr.total_units = unit_base;
+        ctx->stack_sig.swap(sig);
         ctx->stack_valid = true;
-    } else {
-        std::memcpy(&hdr, ctx->stack_host + hdr_off, sizeof hdr);
     }
-    return launch_gemv_stack(ctx, hdr, ctx->stack_dev, batch, (cudaStream_t)stream);
+    return batch == 1 ? launch_gemv1_stack(ctx, ctx->stack_hdr, ctx->stack_dev, st)
+                      : launch_gemv_stack(ctx, ctx->stack_hdr, ctx->stack_dev, batch, st);
 }
 
 int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(const DequantArgs a)
         for (int grp = 0; grp < 2; grp++)
 #pragma unroll
             for (int hr = 0; hr < 2; hr++) {
-                const uint32_t m = __ldg(meta + grp * 16 + g + 8 * hr);
+                const uint32_t m = __ldg(meta + blob_meta_word(grp, g + 8 * hr) / 4);
                 sc[grp][hr] = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
                 zp[grp][hr] = (float)((int)(m >> 16) - a.zero_adjust);
             }

@@ -1,4 +1,5 @@
-// Decode path: fused dequantize-GEMV over tiled field arrays, batch 1..8.
+// Decode path for a batch of 2..8 activation rows: fused dequantize-GEMV over tiled field arrays.
+// (Batch 1 has its own kernel in fq_gemv1.cu.)
 //
 // One persistent CTA per SM with four roles:
 //   producer warp   : streams "units" (32 output rows x one K chunk: every field array of the
@@ -34,6 +35,7 @@
 #include <type_traits>
 
 #include "fq_internal.cuh"
+#include "fq_ptx.cuh"
 
 namespace fq {
 
@@ -61,7 +63,6 @@ constexpr int kOutputWarp = kPrepWarp + kPrepWarps;    // the warp that owns eve
 constexpr int kGemvThreads = (kConsumerWarps + 1 + kPrepWarps + 1) * 32;
 constexpr int kUnitBytes = FQ_GEMV_UNIT_BYTES;         // bytes of one unit (whole blobs), at most: 2 x 4-bit or 1 x 8-bit blob
 constexpr int kXSlots = 3;                             // activation chunks kept in shared memory
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every device-side wait gives up after 2 s
 
 template <int MAXB> struct GemvCfg;
 // kBlobsMax: k blobs (512 columns) per chunk, at most.  kOutSlots: finished units waiting for the output
@@ -143,87 +144,6 @@ static_assert(kUnitBytes >= kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * 8, 
 // A split-K partial is one 64-bit word per (row, batch entry): fp32 sum in the low half, launch tag in the high half.
 size_t gemv_partial_bytes_per_unit(int batch) { return (batch <= 1 ? 32 : 256) * sizeof(unsigned long long); }
 
-// ------------------------------------------------------------------------------- PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait on an mbarrier phase.  Returns false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
-        for (int i = 0; i < 64; i++)
-            if (mbar_try_wait(bar, parity)) return true;      // (no back-off: a sleep here costs 20 % throughput)
-        if (global_ns() - t0 > kWaitLimitNs) return false;
-    }
-}
-// Bounded wait until a condition on shared-memory words written by another warp of this CTA holds.
-template <typename Pred>
-__device__ __forceinline__ bool smem_wait(Pred pred)
-{
-    if (pred()) return true;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
-        for (int i = 0; i < 64; i++) {
-            if (pred()) return true;
-            __nanosleep(20);                       // (a tight spin here takes issue slots from the consumers: -10 %)
-        }
-        if (global_ns() - t0 > kWaitLimitNs) return false;
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v)
-{
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p)
-{
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void red_add_relaxed_u64(unsigned long long* p, unsigned long long v)
-{
-    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p)
-{
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
 // D += A(u8, 16x32, row) * B(s8, 32x8, col), s32 accumulate.
 __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1)
@@ -235,15 +155,7 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 }
 
 // ------------------------------------------------------------------------------- per-CTA work split
-// Units of an op are numbered chunk-major (u = ch * n_rp + rp) and dealt to the CTAs in contiguous
-// blocks; the block boundaries rotate from op to op so that the remainders even out.
-__host__ __device__ __forceinline__ void cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi)
-{
-    const unsigned c = (unsigned)((cta + grid - rot) % grid);
-    lo = (int)((unsigned)n_units * c / (unsigned)grid);              // n_units * grid < 2^31 (checked on the host)
-    hi = (int)((unsigned)n_units * (c + 1u) / (unsigned)grid);
-}
-
+// (this kernel numbers the units of an op chunk-major, u = ch * n_rp + rp, and deals them with cta_range)
 void gemv_cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi) { cta_range(n_units, rot, cta, grid, lo, hi); }
 
 struct StackArgs {
@@ -480,7 +392,7 @@ __device__ __forceinline__ void unit_compute(uint32_t st, int cnt, int blob_read
             int v[TILES][NP][2][2];
             FieldLoop<VARIANT, 0, 0, MAXB, TILES>::run(blob + kBlobMetaBytes + lane * 16, st_tile, xa, (s + ssl) * 256, two_pass, c, v);
             // group epilogue: y += s * 2^-e * (v - z * sum x_int)
-            const uint32_t meta = blob + st_tile * 128 + g * 4;
+            const uint32_t meta = blob + st_tile * 128 + g * 16;          // words of (group, row half) at + group * 8 + half * 4
             if constexpr (MAXB == 1) {
                 // both groups' activation sums and scales in one load each; only the class-0 lane of a quad
                 // subtracts the zero-point term
@@ -489,8 +401,8 @@ __device__ __forceinline__ void unit_compute(uint32_t st, int cnt, int blob_read
                 const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
                 static_for<0, TILES * 2>([&](auto I) {
                     constexpr int tl = decltype(I)::value / 2, grp = decltype(I)::value % 2;
-                    const uint32_t m0 = lds32<tl * 128 + grp * 64>(meta);
-                    const uint32_t m1 = lds32<tl * 128 + grp * 64 + 32>(meta);
+                    const uint32_t m0 = lds32<tl * 128 + grp * 8>(meta);
+                    const uint32_t m1 = lds32<tl * 128 + grp * 8 + 4>(meta);
                     const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
                     const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
                     // v - (z - adjust) * X  =  v + z * (-X) - adjust * (-X)
@@ -505,8 +417,8 @@ __device__ __forceinline__ void unit_compute(uint32_t st, int cnt, int blob_read
                 for (int tl = 0; tl < TILES; tl++) {
 #pragma unroll
                     for (int grp = 0; grp < 2; grp++) {
-                        const uint32_t m0 = lds32(meta + tl * 128 + grp * 64);
-                        const uint32_t m1 = lds32(meta + tl * 128 + grp * 64 + 32);
+                        const uint32_t m0 = lds32(meta + tl * 128 + grp * 8);
+                        const uint32_t m1 = lds32(meta + tl * 128 + grp * 8 + 4);
                         const float s0 = __low2float(*reinterpret_cast<const __half2*>(&m0));
                         const float s1 = __low2float(*reinterpret_cast<const __half2*>(&m1));
                         const int z0 = (int)(m0 >> 16) - kAdjust;
@@ -1114,7 +1026,7 @@ int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st)
     sa.n_phases = 0;
     sa.epoch = next_epoch(ctx->launch_epoch);
     const long long units = (long long)op.n_rp * op.n_chunks;
-    return op.batch <= 1 ? launch_impl<1>(ctx, op, sa, units, st) : launch_impl<8>(ctx, op, sa, units, st);
+    return launch_impl<8>(ctx, op, sa, units, st);
 }
 
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st)
@@ -1131,48 +1043,8 @@ int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, i
     sa.n_phases = hdr.n_phases;
     sa.epoch = next_epoch(ctx->launch_epoch);
     GemvOp dummy{};
-    return max_batch <= 1 ? launch_impl<1>(ctx, dummy, sa, hdr.total_units, st)
-                          : launch_impl<8>(ctx, dummy, sa, hdr.total_units, st);
-}
-
-// ------------------------------------------------------------------------------- allocation-free variant
-// Split-K scratch that is part of the library image, for callers that must not allocate.
-// Host code may only use the symbol through cudaGetSymbolAddress (its name is not a device
-// address on the host side).
-static __device__ __align__(256) unsigned char g_static_scratch[FQ_STATIC_SCRATCH_BYTES];
-
-static int static_scratch_address(int device, unsigned char** out)
-{
-    static unsigned char* addr[64] = {};
-    if (device < 0 || device >= 64) return FQ_ERR_ARG;
-    if (!addr[device]) {                       // once per device, with that device current
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return FQ_ERR_CUDA;
-        addr[device] = static_cast<unsigned char*>(p);
-    }
-    *out = addr[device];
-    return FQ_OK;
-}
-
-// Runs one batch-1 decode op with its split-K partials placed in the built-in array.
-// The array keeps the previous call's contents.  Nothing in it has to start at zero: a partial is
-// only believed when it carries this call's tag, and the tags of the calls that share the array
-// (all contexts on a device) come from one counter per device.
-int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st)
-{
-    static unsigned epoch[64] = {};
-    if (partial_bytes > FQ_STATIC_SCRATCH_BYTES) return FQ_ERR_SCRATCH;
-    unsigned char* base = nullptr;
-    const int rc = static_scratch_address(ctx->device, &base);
-    if (rc != FQ_OK) return rc;
-    op.partial = reinterpret_cast<unsigned long long*>(base);
-    StackArgs sa{};
-    sa.table = nullptr;
-    sa.status = ctx->status_dev;
-    sa.n_ops = 1;
-    sa.n_phases = 0;
-    sa.epoch = next_epoch(epoch[ctx->device]);
-    return launch_impl<1>(ctx, op, sa, (long long)op.n_rp * op.n_chunks, st);
+    (void)max_batch;
+    return launch_impl<8>(ctx, dummy, sa, hdr.total_units, st);
 }
 
 }  // namespace fq

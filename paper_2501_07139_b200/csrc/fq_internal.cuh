@@ -69,16 +69,23 @@ struct Ctx {
     // stack-call staging
     char* stack_dev = nullptr;   // device copy of the op table
     size_t stack_dev_bytes = 0;
-    char* stack_host = nullptr;  // pinned
-    size_t stack_host_bytes = 0;
     // prefill: dequantised bf16 copy of the layer being multiplied
     char* gemm_ws = nullptr;
     size_t gemm_ws_bytes = 0;
     std::vector<void*> owned;    // device buffers allocated by fq_load, freed by fq_destroy
     uint64_t config_epoch = 0;
     unsigned launch_epoch = 0;   // tag of the split-K partials of the latest decode launch (never 0)
-    uint64_t stack_key = 0;      // hash of the op list that is currently uploaded
+    // the op list that is currently uploaded: every argument word of the call that built it
+    std::vector<uint64_t> stack_sig;
     bool stack_valid = false;
+    StackHeader stack_hdr{};
+    // pinned staging buffers of the op table take turns; an event per buffer marks the end of its last upload
+    char* stage_host[2] = {nullptr, nullptr};
+    size_t stage_host_bytes[2] = {0, 0};
+    cudaEvent_t stage_done[2] = {nullptr, nullptr};
+    int stage_next = 0;
+    size_t ws_reserved = 0;      // split-K bytes that the registered layers need (each used once per launch)
+    unsigned long long wait_limit_ns = 2000000000ull;   // limit of every device-side wait
 };
 
 // Bytes of device workspace for `n_ops` ops whose split-K needs are summed by the caller.
@@ -99,12 +106,52 @@ int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, 
 // Chunking policy of the decode kernel: k blobs (512 columns) per K chunk.
 int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_bytes_per_unit(int batch);
-int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);
+int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                 // batch 2..8
+int launch_gemv1_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                // batch 1
+// table_dev: [GemvOp x n_ops][int phase_total x max(n_phases,1)]
+int launch_gemv1_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, cudaStream_t st);
+int gemv1_max_phases();
+int gemv1_max_k();
 int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st);
 // table_dev: [GemvOp x n_ops][long long phase_total x max(n_phases,1)][int cta_units x sm_count]
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
 // Units of an op (n_units units, block rotation rot) that CTA `cta` of `grid` processes: [lo, hi).
 void gemv_cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi);
+
+// ---- how a decode op is dealt to the CTAs of the persistent grid (shared by host and device code)
+// Units of an op (one unit = one K chunk of one 32-row strip) are numbered strip-major, u = rp * n_chunks + ch,
+// and dealt in contiguous blocks; the block boundaries rotate from op to op so that the remainders even out.
+FQ_HD void cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi)
+{
+    const unsigned c = (unsigned)((cta + grid - rot) % grid);
+    lo = (int)((unsigned)n_units * c / (unsigned)grid);              // n_units * grid < 2^31 (checked on the host)
+    hi = (int)((unsigned)n_units * (c + 1u) / (unsigned)grid);
+}
+// The strips a CTA touches: rp_first .. rp_last; only the first may start and only the last may end inside a strip.
+struct CtaWork {
+    int lo, hi, rp_first, rp_last;
+    FQ_HD bool any() const { return hi > lo; }
+    // chunks [c0, c1) of strip rp that belong to this CTA
+    FQ_HD void chunks(int n_chunks, int rp, int& c0, int& c1) const
+    {
+        c0 = rp == rp_first ? lo - rp * n_chunks : 0;
+        c1 = rp == rp_last ? hi - rp * n_chunks : n_chunks;
+    }
+    // strips that this CTA finishes (it owns their last chunk) and therefore writes to y
+    FQ_HD int finishing(int n_chunks) const
+    {
+        if (!any()) return 0;
+        return rp_last - rp_first + 1 - (hi - rp_last * n_chunks < n_chunks ? 1 : 0);
+    }
+};
+FQ_HD CtaWork cta_work(int n_units, int n_chunks, int rot, int cta, int grid)
+{
+    CtaWork w;
+    cta_range(n_units, rot, cta, grid, w.lo, w.hi);
+    w.rp_first = w.lo / n_chunks;
+    w.rp_last = w.hi > w.lo ? (w.hi - 1) / n_chunks : w.rp_first;
+    return w;
+}
 
 int launch_gemm(Ctx* ctx, const void* store, int blob_stride, const FieldList& fl, int zero_adjust, int n_out, int k_in,
                 const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, void* w_scratch, cudaStream_t st);

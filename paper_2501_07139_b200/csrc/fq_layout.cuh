@@ -7,7 +7,8 @@
 //                   so a b-bit child is the first b-1 arrays = the first b/8 of the bytes.
 // Storage is cut into BLOBS: one blob = one row pair (32 rows = two 16-row tiles) x 512 columns
 // (two "supersteps" of 256).  A blob holds, in this order,
-//     scale/zero words   [superstep][tile][group][16 rows]                       (512 B)
+//     scale/zero words   [superstep][tile][row & 7][group][row >> 3]             (512 B)
+//                        (the four words that one lane of the decode kernel needs are one 16-byte load)
 //     field array 0      [superstep][tile][f0 chunks][32 lanes][16 B]            (2048 * f0 B)
 //     field array 1 ...                                                          (most significant first)
 // and blobs are ordered [row_pair][k_blob].  Everything a decode unit needs is therefore ONE
@@ -97,6 +98,8 @@ FQ_HD int64_t store_bytes(int n_out, int k_in, int bits) { return (int64_t)row_p
 // Offsets inside a blob: scale/zero words of (superstep ssl, tile), and the tile of field width f
 // that comes after fields adding up to prefix_bits.
 FQ_HD int blob_meta_off(int ssl, int tile) { return (ssl * kBlobTiles + tile) * 128; }
+// ... and inside that, the word of row r (0..15) of the tile and group grp (0..1) of the superstep
+FQ_HD int blob_meta_word(int grp, int r) { return (r & 7) * 16 + grp * 8 + (r >> 3) * 4; }
 FQ_HD int blob_field_off(int prefix_bits, int f, int ssl, int tile)
 {
     return kBlobMetaBytes + kBlobSteps * kBlobTiles * 512 * prefix_bits + (ssl * kBlobTiles + tile) * f * 512;

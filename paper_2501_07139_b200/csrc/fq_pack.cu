@@ -114,8 +114,8 @@ __global__ void __launch_bounds__(256) pack_kernel(const StoreArgs a)
         const int rp = (int)(blob / a.n_kb), kb = (int)(blob % a.n_kb);
         unsigned v = 0;
         if (off < kBlobMetaBytes) {
-            // scale/zero word: [superstep][tile][group][16 rows]
-            const int r = (off >> 2) & 15, grp = (off >> 6) & 1, tile = (off >> 7) & 1, ssl = off >> 8;
+            // scale/zero word: [superstep][tile][row & 7][group][row >> 3]
+            const int r = ((off >> 4) & 7) + 8 * ((off >> 2) & 1), grp = (off >> 3) & 1, tile = (off >> 7) & 1, ssl = off >> 8;
             const long long n = ((long long)rp * kBlobTiles + tile) * kTileRows + r;
             const int g = (kb * kBlobSteps + ssl) * 2 + grp;
             if (n < a.n_out && g < a.groups) {
@@ -250,8 +250,8 @@ __global__ void __launch_bounds__(256) export_meta_kernel(const ExportArgs a)
         const int g = (int)(i % a.groups);
         int tile, ssl;
         const uint8_t* blob = blob_of(a, n, (long long)g * kGroup, tile, ssl);
-        const uint32_t v = *reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile) + (g & 1) * 64 +
-                                                              (int)(n % kTileRows) * 4);
+        const uint32_t v = *reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile) +
+                                                              blob_meta_word(g & 1, (int)(n % kTileRows)));
         a.scales[i] = (uint16_t)(v & 0xffffu);
         a.zeros[i] = __half_as_ushort(__float2half_rn((float)(v >> 16)));
     }
