@@ -71,13 +71,14 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.n_ss = supersteps(L.k_in);
     op.n_kb = k_blobs(L.k_in);
     op.n_rp = row_pairs(L.n_out);
-    op.chunk_blobs = gemv_chunk_blobs(bits, batch);
+    op.chunk_blobs = batch == 1 ? gemv1_chunk_blobs(op.blob_read) : gemv_chunk_blobs(bits, batch);
     op.n_chunks = (op.n_kb + op.chunk_blobs - 1) / op.chunk_blobs;
     op.batch = batch;
     // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
     op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
-    op.n_units = op.n_chunks * op.n_rp;
-    if ((long long)op.n_chunks * op.n_rp * 1024 >= (1ll << 31)) return FQ_ERR_SHAPE;   // 32-bit unit arithmetic on the device
+    // what is dealt to the CTAs: batch 1 the blobs of every strip, batch 2..8 the K chunks of every row pair
+    op.n_units = (batch == 1 ? op.n_kb : op.n_chunks) * op.n_rp;
+    if ((long long)op.n_units * 1024 >= (1ll << 31)) return FQ_ERR_SHAPE;              // 32-bit unit arithmetic on the device
     if (batch == 1 && L.k_in > gemv1_max_k()) return FQ_ERR_SHAPE;                   // a strip's activations stay in shared memory
     op.phase = -1;
     op.rot = 0;
@@ -88,8 +89,8 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
 // share are ever written.  Batch 2..8: one tagged word per (row pair, K chunk, row, batch entry).
 size_t op_partial_bytes(const GemvOp& op, int max_batch)
 {
+    if (max_batch <= 1) return op.n_kb <= 1 ? 0 : (size_t)op.n_rp * op.n_kb * 32 * sizeof(unsigned long long);
     if (op.n_chunks <= 1) return 0;
-    if (max_batch <= 1) return (size_t)op.n_rp * op.n_kb * 32 * sizeof(unsigned long long);
     return (size_t)op.n_rp * op.n_chunks * gemv_partial_bytes_per_unit(max_batch);
 }
 
@@ -504,11 +505,13 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         sig.push_back(phases_host ? (uint64_t)(int64_t)phases_host[i] : 0u);
     }
     const int np = n_phases > 0 ? n_phases : 1;
-    // batch 1:    [GemvOp x n_ops][int phase_total x np]
+    // batch 1:    [GemvOp x n_ops][int phase_total x np][uint2 strips x sm_count x n_ops]
     // batch 2..8: [GemvOp x n_ops][long long phase_total x np][int cta_units x sm_count]
-    const size_t table_bytes = (size_t)n_ops * sizeof(GemvOp) +
-                               (batch == 1 ? (size_t)np * sizeof(int)
-                                           : (size_t)np * sizeof(long long) + (size_t)ctx->sm_count * sizeof(int));
+    const size_t range_off = (size_t)round_up((int64_t)((size_t)n_ops * sizeof(GemvOp) + (size_t)np * sizeof(int)), 8);
+    const size_t table_bytes = batch == 1 ? range_off + (size_t)ctx->sm_count * n_ops * sizeof(uint2)
+                                          : (size_t)n_ops * sizeof(GemvOp) + (size_t)np * sizeof(long long) +
+                                                (size_t)ctx->sm_count * sizeof(int);
+    if (batch == 1 && n_ops > gemv1_max_ops()) return FQ_ERR_SHAPE;
 
     if (!(ctx->stack_valid && ctx->stack_sig == sig)) {
         ctx->stack_valid = false;                           // until the new table is complete
@@ -548,15 +551,45 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             // per phase: CTAs that finish at least one strip (each reports once when its strips are done)
             int* phase_total = reinterpret_cast<int*>(host + (size_t)n_ops * sizeof(GemvOp));
             for (int p = 0; p < np; p++) phase_total[p] = 0;
-            if (phases_host) {
-                std::vector<int> last_phase(grid, -1);
-                for (int i = 0; i < n_ops; i++)
-                    for (int c = 0; c < grid; c++)
-                        if (cta_work(ops[i].n_units, ops[i].n_chunks, ops[i].rot, c, grid).finishing(ops[i].n_chunks) > 0 &&
-                            last_phase[c] != phases_host[i]) {
+            // ... and for every (CTA, op) the strips the CTA computes.  The ops of one dependency phase (of the
+            // whole list when there are no phases) are dealt together: their blobs form one sequence, op
+            // after op, and every CTA gets the same number of BYTES of it in one contiguous piece.  A CTA
+            // then touches one or two ops of a phase instead of all of them: fewer activation vectors to
+            // convert, fewer strips shared with a neighbour.
+            uint2* ranges = reinterpret_cast<uint2*>(host + range_off);
+            std::vector<int> last_phase(grid, -1);
+            for (int g0 = 0, group = 0; g0 < n_ops; group++) {
+                int g1 = g0 + 1;
+                while (g1 < n_ops && (!phases_host || phases_host[g1] == phases_host[g0])) g1++;
+                unsigned long long total = 0;
+                for (int i = g0; i < g1; i++) total += (unsigned long long)ops[i].n_units * (unsigned)ops[i].blob_read;
+                const int rot = (int)((unsigned)group * 53u % (unsigned)grid);      // spreads the remainders
+                unsigned long long before = 0;
+                for (int i = g0; i < g1; i++) {
+                    const unsigned long long sz = (unsigned)ops[i].blob_read;
+                    const unsigned long long bytes = (unsigned long long)ops[i].n_units * sz;
+                    for (int c = 0; c < grid; c++) {
+                        const unsigned long long cc = (unsigned)((c + grid - rot) % grid);
+                        // blobs of this op whose first byte lies in [cut(cc), cut(cc + 1))
+                        auto first_blob_at = [&](unsigned long long pos) -> long long {
+                            if (pos <= before) return 0;
+                            if (pos >= before + bytes) return ops[i].n_units;
+                            return (long long)((pos - before + sz - 1) / sz);
+                        };
+                        CtaWork w;
+                        w.lo = (int)first_blob_at(total * cc / (unsigned)grid);
+                        w.hi = (int)first_blob_at(total * (cc + 1) / (unsigned)grid);
+                        w.rp_first = w.lo / ops[i].n_kb;
+                        w.rp_last = w.hi > w.lo ? (w.hi - 1) / ops[i].n_kb : w.rp_first;
+                        ranges[(size_t)c * n_ops + i] = gemv1_pack_range(w, ops[i].n_kb);
+                        if (phases_host && w.finishing(ops[i].n_kb) > 0 && last_phase[c] != phases_host[i]) {
                             last_phase[c] = phases_host[i];
                             phase_total[phases_host[i]]++;
                         }
+                    }
+                    before += bytes;
+                }
+                g0 = g1;
             }
         } else {
             long long* phase_total = reinterpret_cast<long long*>(host + (size_t)n_ops * sizeof(GemvOp));

@@ -1,13 +1,14 @@
 // Decode path, batch 1: fused dequantize-GEMV over tiled field arrays, one persistent CTA per SM.
 //
-// Work split.  An op (one matrix) is cut into STRIPS of 32 output rows x the whole K, a strip into K
-// chunks ("units": 1..3 blobs of 512 columns, what one ring stage holds).  Units are numbered strip-major
-// and dealt to the CTAs in equal contiguous blocks (cta_work in fq_internal.cuh), so every CTA streams the
-// same number of bytes and almost every strip is computed by ONE CTA from end to end: its K reduction
-// stays in shared memory and the CTA writes y itself.  Only a strip that a block boundary cuts is shared
-// by two (rarely three) CTAs: the CTA that owns the strip's last chunk finishes it, the others publish the
-// sums of their blobs as tagged 64-bit words (fp32 value, launch tag) in global memory and process that
-// strip first, long before the finisher asks for them.  y[row] is always the sum of the per-blob sums in
+// Work split.  An op (one matrix) is cut into STRIPS of 32 output rows x the whole K, a strip into blobs of
+// 512 columns.  Blobs are numbered strip-major and dealt to the CTAs in equal contiguous blocks (cta_work in
+// fq_internal.cuh), so every CTA streams the same number of bytes and almost every strip is computed by ONE
+// CTA from end to end: its K reduction stays in shared memory and the CTA writes y itself.  Only a strip
+// that a block boundary cuts is shared by two (rarely three) CTAs: the CTA that owns the strip's FIRST blob
+// finishes it, the others publish the sums of their blobs as tagged 64-bit words (fp32 value, launch tag)
+// in global memory.  The shared strip is the last thing the finisher computes and the first thing the
+// publisher computes, so the words are there long before they are asked for.  A CTA streams
+// its blobs of a strip in "units" of up to six (what one ring stage holds).  y[row] is always the sum of the per-blob sums in
 // blob order, whoever computed them, so results do not depend on how the op was dealt.
 //
 // Roles of a CTA:
@@ -41,15 +42,17 @@ constexpr int kCW = 16;                                // consumer warps: K lane
 constexpr int kKLanes = kCW / kBlobTiles;
 constexpr int kProducerWarp = kCW;
 constexpr int kPrepWarp = kCW + 1;                     // first activation pre-processing warp
-constexpr int kPrepWarps = 4;
+constexpr int kPrepWarps = 8;
 constexpr int kThreads = (kCW + 1 + kPrepWarps) * 32;
-constexpr int kStageBytes = 17408;                     // one unit: 2 x 4-bit blobs or 1 x 8-bit blob
-constexpr int kBlobsMax = 3;                           // blobs per unit, at most
+constexpr int kStageBytes = 34816;                     // one unit: 4 x 4-bit blobs or 2 x 8-bit blobs
+constexpr int kBlobsMax = 6;                           // blobs per unit, at most (< kKLanes: a warp gets at most one item of a unit)
 constexpr int kXSlots = 32;                            // activation blobs resident in shared memory
 constexpr int kStripSlots = 4;                         // strips whose items are in flight
-constexpr int kMaxKb = 32;                             // blobs per strip, at most (k_in <= 16384)
+constexpr int kMaxKb = 28;                             // blobs per strip, at most (k_in <= 14336)
 constexpr int kQD = 8;                                 // entries per consumer queue
 constexpr int kMaxPhasesDev = 1024;
+constexpr int kMaxOpsDev = 512;                        // ops of one launch (their per-CTA ranges sit in shared memory)
+static_assert(kXSlots % kPrepWarps == 0, "an activation slot is always filled by the same warp");
 
 // What the producer tells a consumer warp about one item (one 16-byte store, one 16-byte load).
 //   w0 blob shared address   w1 packed fields (below)   w2 activation blob number + 1   w3 sequence tag
@@ -66,7 +69,7 @@ struct StripDesc {
     unsigned long long* partial;             // tagged blob sums of this strip in global memory: [blob][32 rows]
     int n_out, row_base;
     int n_kb, kb_lo, kb_hi;                  // blobs of the strip; [kb_lo, kb_hi) are computed by this CTA
-    int finish;                              // this CTA owns the last chunk: it adds up and writes y
+    int finish;                              // this CTA owns the first blob: it adds up and writes y
     int phase;
     int expect;                              // items of this CTA in the strip
     int pad[4];
@@ -75,7 +78,7 @@ static_assert(sizeof(StripDesc) == 64, "descriptor layout");
 
 struct Smem {
     static constexpr int kFixed = kXSlots * (kXBlobDigitBytes + kXBlobGroupBytes) + 1024 + kStripSlots * kMaxKb * 128 +
-                                  kCW * kQD * 16 + kStripSlots * 64 + kMaxPhasesDev * 2 + 1024;
+                                  kCW * kQD * 16 + kStripSlots * 64 + kMaxPhasesDev + kMaxOpsDev * 8 + 1024;
     static constexpr int kStages = (232448 - kFixed) / kStageBytes;
     static constexpr int oStages = 0;
     static constexpr int oXDig = oStages + kStages * kStageBytes;            // [slot][1024]
@@ -84,8 +87,9 @@ struct Smem {
     static constexpr int oPart = oZero + 1024;                               // float [strip slot][blob][32 rows]
     static constexpr int oQueue = oPart + kStripSlots * kMaxKb * 128;        // uint4 [warp][kQD]
     static constexpr int oStrip = oQueue + kCW * kQD * 16;                   // StripDesc [strip slot]
-    static constexpr int oFinTot = oStrip + kStripSlots * 64;                // u16 [phase]: strips this CTA finishes
-    static constexpr int oBars = oFinTot + kMaxPhasesDev * 2;                // full[S], empty[S]
+    static constexpr int oRange = oStrip + kStripSlots * 64;                 // uint2 [op]: this CTA's strips of every op
+    static constexpr int oFinTot = oRange + kMaxOpsDev * 8;                  // u8 [phase]: strips this CTA finishes
+    static constexpr int oBars = oFinTot + kMaxPhasesDev;                    // full[S], empty[S]
     static constexpr int oCtl = oBars + 2 * 16 * 8;
     // control words (u32 each)
     static constexpr int cXTag = 0;                                          // [kXSlots] activation blob number + 1 held
@@ -93,18 +97,21 @@ struct Smem {
     static constexpr int cStripCnt = cXCnt + kXSlots;                        // [kStripSlots] items delivered
     static constexpr int cStripBusy = cStripCnt + kStripSlots;               // [kStripSlots]
     static constexpr int cFinCnt = cStripBusy + kStripSlots;                 // [8] strips finished, per phase & 7
-    static constexpr int cQn = cFinCnt + 8;                                  // [kCW] entries queued so far (producer only)
-    static constexpr int cAbort = cQn + kCW;
+    static constexpr int cPhaseKnown = cFinCnt + 8;                          // phases 0 .. value - 1 are complete
+    static constexpr int cPollLock = cPhaseKnown + 1;                        // one warp at a time polls the phase counters
+    static constexpr int cAbort = cPollLock + 1;
     static constexpr int kCtlWords = cAbort + 1;
     static constexpr int kTotal = oCtl + kCtlWords * 4;
     static_assert(kStages >= 4 && kStages <= 16, "decode kernel: ring size");
     static_assert(kTotal <= 232448, "decode kernel: shared memory over the 227 KB per-CTA limit");
-    static_assert(oBars % 8 == 0 && oQueue % 16 == 0 && oStrip % 16 == 0 && oXDig % 128 == 0 && oZero % 128 == 0, "alignment");
+    static_assert(oBars % 8 == 0 && oQueue % 16 == 0 && oStrip % 16 == 0 && oXDig % 128 == 0 && oZero % 128 == 0 &&
+                  oRange % 8 == 0, "alignment");
 };
 
 struct Args {
     const GemvOp* table;                   // device op table (nullptr: the by-value op)
     const int* phase_total;                // CTAs that finish at least one strip, per phase
+    const uint2* ranges;                   // [cta][op] strips of every op for every CTA (nullptr: computed here)
     unsigned long long* phase_done;        // CTAs that have finished all their strips, per phase
     unsigned* exit_count;
     int* status;
@@ -132,23 +139,36 @@ __device__ __forceinline__ void sts128(uint32_t a, uint4 v)
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// The strips of one op for one CTA, in the order in which it processes them: a strip that another CTA
-// finishes goes first (its sums are wanted elsewhere), the rest in ascending order.
+// The strips of one op for one CTA: rp_first .. rp_last; the first starts at blob c_first, the last ends
+// before blob c_last (see cta_work).  Packed into two words per (CTA, op) by the host for a stack call.
+constexpr uint32_t kRangeEmpty = 0xffffffffu;
+FQ_HD uint2 pack_range(const CtaWork& w, int n_kb)
+{
+    if (!w.any()) return uint2{kRangeEmpty, 0u};
+    int f0, f1, l0, l1;
+    w.chunks(n_kb, w.rp_first, f0, f1);
+    w.chunks(n_kb, w.rp_last, l0, l1);
+    return uint2{(uint32_t)w.rp_first | (uint32_t)f0 << 20, (uint32_t)w.rp_last | (uint32_t)l1 << 20};
+}
 struct StripOrder {
-    CtaWork w;
-    int n_chunks, n_strips, first_is_last;
-    __device__ __forceinline__ StripOrder(const GemvOp& op, int cta, int grid)
+    int rp_first, rp_last, c_first, c_last, n_kb, n_strips;
+    __device__ __forceinline__ StripOrder(uint2 r, int n_kb_)
     {
-        w = cta_work(op.n_units, op.n_chunks, op.rot, cta, grid);
-        n_chunks = op.n_chunks;
-        n_strips = w.any() ? w.rp_last - w.rp_first + 1 : 0;
-        first_is_last = n_strips > 1 && (w.hi - w.rp_last * n_chunks) < n_chunks;
+        n_kb = n_kb_;
+        if (r.x == kRangeEmpty) { n_strips = 0; rp_first = rp_last = c_first = c_last = 0; return; }
+        rp_first = (int)(r.x & 0xfffffu); c_first = (int)(r.x >> 20);
+        rp_last = (int)(r.y & 0xfffffu); c_last = (int)(r.y >> 20);
+        n_strips = rp_last - rp_first + 1;
     }
-    __device__ __forceinline__ int strip(int i) const
+    __device__ __forceinline__ int strip(int i) const { return rp_first + i; }
+    // blobs [c0, c1) of strip rp that belong to this CTA
+    __device__ __forceinline__ void chunks(int rp, int& c0, int& c1) const
     {
-        if (!first_is_last) return w.rp_first + i;
-        return i == 0 ? w.rp_last : w.rp_first + i - 1;
+        c0 = rp == rp_first ? c_first : 0;
+        c1 = rp == rp_last ? c_last : n_kb;
     }
+    // strips that this CTA finishes (it owns their first blob)
+    __device__ __forceinline__ int finishing() const { return n_strips == 0 ? 0 : n_strips - (c_first > 0 ? 1 : 0); }
 };
 
 __device__ __forceinline__ void raise_timeout(const Args& a, volatile unsigned* ctl)
@@ -251,7 +271,8 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + S::oBars;                               // full[s] at 8 s, empty[s] at 128 + 8 s
     volatile unsigned* ctl = reinterpret_cast<volatile unsigned*>(smem + S::oCtl);
-    unsigned short* fin_total = reinterpret_cast<unsigned short*>(smem + S::oFinTot);
+    unsigned char* fin_total = smem + S::oFinTot;
+    const uint2* range = reinterpret_cast<const uint2*>(smem + S::oRange);
     const GemvOp* ops = a.table ? a.table : &single;
 
     if (threadIdx.x == 0) {
@@ -265,101 +286,129 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
     for (int i = threadIdx.x; i < S::kCtlWords; i += blockDim.x) ctl[i] = 0u;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + S::oZero)[i] = 0u;
     for (int i = threadIdx.x; i < kCW * kQD * 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + S::oQueue)[i] = 0u;
-    for (int i = threadIdx.x; i < kMaxPhasesDev / 2; i += blockDim.x) reinterpret_cast<uint32_t*>(fin_total)[i] = 0u;
+    for (int i = threadIdx.x; i < kMaxPhasesDev / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(fin_total)[i] = 0u;
+    // this CTA's strips of every op
+    for (int oi = threadIdx.x; oi < a.n_ops; oi += blockDim.x) {
+        uint2 r;
+        if (a.ranges) r = a.ranges[(long long)cta * a.n_ops + oi];
+        else r = pack_range(cta_work(ops[oi].n_units, ops[oi].n_kb, ops[oi].rot, cta, grid), ops[oi].n_kb);
+        reinterpret_cast<uint2*>(smem + S::oRange)[oi] = r;
+    }
     __syncthreads();
     // strips that this CTA finishes, per phase (the warp that finishes the last one reports the phase)
     if (a.n_phases > 0) {
         for (int oi = threadIdx.x; oi < a.n_ops; oi += blockDim.x) {
-            const GemvOp& op = ops[oi];
-            const int fin = cta_work(op.n_units, op.n_chunks, op.rot, cta, grid).finishing(op.n_chunks);
-            if (fin > 0 && op.phase >= 0) {
-                // two 16-bit counters per word
-                atomicAdd(reinterpret_cast<unsigned*>(fin_total) + (op.phase >> 1), (unsigned)fin << (16 * (op.phase & 1)));
-            }
+            const int phase = ops[oi].phase;
+            const int fin = StripOrder(range[oi], ops[oi].n_kb).finishing();
+            if (fin > 0 && phase >= 0)                              // four 8-bit counters per word
+                atomicAdd(reinterpret_cast<unsigned*>(fin_total) + (phase >> 2), (unsigned)fin << (8 * (phase & 3)));
         }
     }
     __syncthreads();
 
     if (warp == kProducerWarp) {
         // ================================================================== producer
+        // This loop is the serial path that feeds the whole CTA: per unit it costs lane 0 a barrier test, the
+        // transaction count, one bulk copy and one arrival; the item descriptors are written by the lanes of
+        // the warps they are meant for (lane w keeps the number of entries queued for consumer warp w).
         int stage = 0;
         unsigned wraps = 0;
         unsigned rr = 0;                              // K lane of the next blob (round-robin over everything)
         unsigned xseq = 0;                            // activation blobs of the ops seen so far
         unsigned strip_seq = 0;
+        unsigned qn = 0;                              // lane w < kCW: entries queued for consumer warp w
         bool stop = false;
-        StripDesc* sdesc = reinterpret_cast<StripDesc*>(smem + S::oStrip);
+        const uint32_t sdesc_a = sbase + S::oStrip;
+        const unsigned long long stream_policy = l2_policy_evict_first();      // weights are read once per pass
+        const uint32_t my_queue = sbase + S::oQueue + (uint32_t)(lane & (kCW - 1)) * kQD * 16u;
+        const int my_klane = (lane >> 1) & (kKLanes - 1), my_tile = lane & 1;
+        // The descriptor of the next op travels while the units of the current one are issued.
+        struct OpRegs {
+            const uint8_t* store;
+            unsigned long long* partial;
+            uint16_t* y;
+            int blob_read, blob_stride, n_kb, cb, variant, n_out, phase;
+            __device__ __forceinline__ void fetch(const GemvOp* ops, int oi, int n_ops)
+            {
+                if (oi >= n_ops) return;
+                const GemvOp& o = ops[oi];
+                store = o.store; partial = o.partial; y = o.y; blob_read = o.blob_read; blob_stride = o.blob_stride;
+                n_kb = o.n_kb; cb = o.chunk_blobs; variant = o.variant; n_out = o.n_out; phase = o.phase;
+            }
+        };
+        OpRegs nxt;
+        nxt.fetch(ops, 0, a.n_ops);
         for (int oi = 0; oi < a.n_ops && !stop; oi++) {
-            prefetch_ops(ops, oi, a.n_ops, lane);
-            const GemvOp& op = ops[oi];
-            const StripOrder so(op, cta, grid);
+            const OpRegs cur = nxt;
+            nxt.fetch(ops, oi + 1, a.n_ops);
+            const int n_kb = cur.n_kb, cb = cur.cb, variant = cur.variant, n_out = cur.n_out, phase = cur.phase;
+            const StripOrder so(range[oi], n_kb);
             if (so.n_strips == 0) continue;
-            const int n_kb = op.n_kb, cb = op.chunk_blobs;
-            const uint32_t blob_read = (uint32_t)op.blob_read;
-            const long long blob_stride = op.blob_stride;
-            const bool contiguous = op.blob_read == op.blob_stride;
+            const uint32_t blob_read = (uint32_t)cur.blob_read;
+            const long long blob_stride = cur.blob_stride;
+            const uint8_t* const store = cur.store;
+            uint16_t* const y = cur.y;
+            unsigned long long* const partial = cur.partial;
+            const bool contiguous = cur.blob_read == cur.blob_stride;
             for (int si = 0; si < so.n_strips && !stop; si++) {
                 const int rp = so.strip(si);
                 int c0, c1;
-                so.w.chunks(so.n_chunks, rp, c0, c1);
-                const int kb_lo = c0 * cb, kb_hi = min(c1 * cb, n_kb);
+                so.chunks(rp, c0, c1);
+                const int kb_lo = c0, kb_hi = c1;
                 const int sslot = (int)(strip_seq % kStripSlots);
                 strip_seq++;
                 int slot_ok = 1;
-                if (lane == 0) {
-                    if (!wait_smem([&] { return ctl[S::cStripBusy + sslot] == 0u; }, ctl, a.wait_ns)) {
-                        if (!ctl[S::cAbort]) raise_timeout(a, ctl);
-                        slot_ok = 0;
-                    } else {
-                        StripDesc& d = sdesc[sslot];
-                        d.y = op.y;
-                        d.partial = op.partial + (long long)rp * n_kb * 32;
-                        d.n_out = op.n_out; d.row_base = rp * (kBlobTiles * kTileRows);
-                        d.n_kb = n_kb; d.kb_lo = kb_lo; d.kb_hi = kb_hi;
-                        d.finish = c1 == so.n_chunks;
-                        d.phase = op.phase;
-                        d.expect = (kb_hi - kb_lo) * kBlobTiles;
-                        ctl[S::cStripBusy + sslot] = 1u;
-                        __threadfence_block();
-                    }
+                if (lane == 0 && !wait_smem([&] { return ctl[S::cStripBusy + sslot] == 0u; }, ctl, a.wait_ns)) {
+                    if (!ctl[S::cAbort]) raise_timeout(a, ctl);
+                    slot_ok = 0;
                 }
                 if (!__shfl_sync(0xffffffffu, slot_ok, 0)) { stop = true; break; }   // (every loop exit is decided by lane 0)
-                const uint8_t* src = op.store + ((long long)rp * n_kb + kb_lo) * blob_stride;
+                {
+                    // the strip's descriptor: three lanes store 16 bytes each
+                    unsigned long long* const sp = partial + (long long)rp * n_kb * 32;
+                    uint4 d;
+                    if (lane == 0) d = make_uint4((uint32_t)(uintptr_t)y, (uint32_t)((uintptr_t)y >> 32), (uint32_t)(uintptr_t)sp,
+                                                  (uint32_t)((uintptr_t)sp >> 32));
+                    else if (lane == 1) d = make_uint4((uint32_t)n_out, (uint32_t)(rp * (kBlobTiles * kTileRows)), (uint32_t)n_kb, (uint32_t)kb_lo);
+                    else d = make_uint4((uint32_t)kb_hi, c0 == 0 ? 1u : 0u, (uint32_t)phase, (uint32_t)((kb_hi - kb_lo) * kBlobTiles));
+                    if (lane < 3) sts128(sdesc_a + (uint32_t)sslot * 64u + (uint32_t)lane * 16u, d);
+                    if (lane == 0) ctl[S::cStripBusy + sslot] = 1u;
+                    __threadfence_block();                           // the descriptor before any item that refers to it
+                    __syncwarp();
+                }
+                const uint8_t* src = store + ((long long)rp * n_kb + kb_lo) * blob_stride;
                 for (int kb = kb_lo; kb < kb_hi; kb += cb) {
                     const int nb = min(cb, kb_hi - kb);
                     const uint32_t full = bars + 8 * stage, empty = bars + 128 + 8 * stage;
+                    const uint32_t stage_base = sbase + S::oStages + (uint32_t)stage * kStageBytes;
                     int ok = 1;
                     if (lane == 0) {
                         if (wraps > 0 && !wait_mbar(empty, (wraps - 1u) & 1u, ctl, a.wait_ns)) {
                             if (!ctl[S::cAbort]) raise_timeout(a, ctl);
                             ok = 0;
                         }
-                        if (ok) mbar_expect_tx(full, (uint32_t)nb * blob_read);
+                        if (ok) {
+                            mbar_expect_tx(full, (uint32_t)nb * blob_read);
+                            if (contiguous) bulk_g2s_hint(stage_base, src, (uint32_t)nb * blob_read, full, stream_policy);
+                            mbar_arrive_n(empty, (uint32_t)(kCW - nb * kBlobTiles));   // for the warps without an item in this unit
+                        }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) { stop = true; break; }
-                    const uint32_t stage_base = sbase + S::oStages + (uint32_t)stage * kStageBytes;
-                    if (contiguous) {
-                        if (lane == 0) bulk_g2s(stage_base, src, (uint32_t)nb * blob_read, full);
-                    } else if (lane < nb) {
-                        bulk_g2s(stage_base + lane * blob_read, src + lane * blob_stride, blob_read, full);
-                    }
-                    // the items of this unit: lane = blob * 2 + tile
-                    if (lane < nb * kBlobTiles) {
-                        const int b = lane >> 1, t = lane & 1;
-                        const int w = (int)(((rr + (unsigned)b) % kKLanes) * kBlobTiles) + t;
-                        const unsigned n = ctl[S::cQn + w];
+                    if (!contiguous && lane < nb) bulk_g2s_hint(stage_base + lane * blob_read, src + lane * blob_stride, blob_read, full, stream_policy);
+                    // the items of this unit: blob b goes to K lane (rr + b) mod 8, its two tiles to that lane's two warps
+                    const int b = (int)((unsigned)my_klane - rr) & (kKLanes - 1);
+                    if (lane < kCW && b < nb) {
                         const unsigned xs = xseq + (unsigned)(kb + b);
                         uint4 e;
                         e.x = stage_base + (uint32_t)b * blob_read;
-                        e.y = item_pack((int)(xs % kXSlots), stage, (int)(wraps & 1u), kb + b, sslot, op.variant);
+                        e.y = item_pack((int)(xs % kXSlots), stage, (int)(wraps & 1u), kb + b, sslot, variant);
                         e.z = xs + 1u;
-                        e.w = n + 1u;
-                        sts128(sbase + S::oQueue + (uint32_t)(w * kQD + (int)(n % kQD)) * 16u, e);
-                        ctl[S::cQn + w] = n + 1u;
+                        e.w = qn + 1u;
+                        sts128(my_queue + (qn % kQD) * 16u, e);
+                        qn++;
                     }
-                    if (lane == 0) mbar_arrive_n(empty, (uint32_t)(kCW - nb * kBlobTiles));   // warps without an item in this unit
-                    __syncwarp();
+                    (void)my_tile;
                     rr += (unsigned)nb;
                     src += (long long)nb * blob_stride;
                     if (++stage == S::kStages) { stage = 0; wraps++; }
@@ -369,11 +418,9 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         }
         // the end marker of every queue
         if (lane < kCW) {
-            const unsigned n = ctl[S::cQn + lane];
-            const uint4 e = make_uint4(0u, kItemEnd, 0u, n + 1u);
             // (the queue slot is free: a warp gets one entry per kKLanes blobs, so the entry that used the slot
             // kQD entries ago belongs to a unit whose stage has been refilled since, i.e. it was consumed)
-            sts128(sbase + S::oQueue + (uint32_t)(lane * kQD + (int)(n % kQD)) * 16u, e);
+            sts128(my_queue + (qn % kQD) * 16u, make_uint4(0u, kItemEnd, 0u, qn + 1u));
         }
         // copies that are still in flight must land before the CTA may exit
         if (stop && lane == 0) {
@@ -385,90 +432,134 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         }
     } else if (warp >= kPrepWarp) {
         // ================================================================== activation pre-processing
+        // The activation blobs of all ops this CTA takes part in form one sequence; warp pw converts the blobs
+        // whose number is congruent to pw.  The loads of a warp's next blob travel while it converts the
+        // current one; they are only issued once the op's phase is known to be open.
         const int pw = warp - kPrepWarp;
-        unsigned xseq = 0;
-        int phase_known = -1;                         // every phase <= phase_known is complete
-        bool stop = false;
-        for (int oi = 0; oi < a.n_ops && !stop; oi++) {
-            prefetch_ops(ops, oi, a.n_ops, lane);
-            const GemvOp& op = ops[oi];
-            const StripOrder so(op, cta, grid);
-            if (so.n_strips == 0) continue;
-            const int n_kb = op.n_kb, cb = op.chunk_blobs;
-            // blobs of x that this CTA's strips cover: the first and the last strip may be partial
-            int f0, f1, l0, l1;
-            so.w.chunks(so.n_chunks, so.w.rp_first, f0, f1);
-            so.w.chunks(so.n_chunks, so.w.rp_last, l0, l1);
-            const int fk0 = f0 * cb, fk1 = min(f1 * cb, n_kb), lk0 = l0 * cb, lk1 = min(l1 * cb, n_kb);
-            const int n_mid = so.n_strips > 2 ? so.n_strips - 2 : 0;
-            // the activations are the previous phase's outputs
-            if (op.phase > 0 && phase_known < op.phase - 1) {
-                int ok = 1;
-                if (lane == 0) {
-                    const unsigned long long need = (unsigned long long)a.phase_total[op.phase - 1];
-                    const unsigned long long t0 = global_ns();
-                    unsigned it = 0;
-                    while (ld_acquire_u64(a.phase_done + (op.phase - 1)) < need) {
-                        if ((++it & 31u) == 0u) {
-                            if (ctl[S::cAbort]) { ok = 0; break; }
-                            if (global_ns() - t0 > a.wait_ns || *reinterpret_cast<volatile int*>(a.status) != 0) {
-                                raise_timeout(a, ctl); ok = 0; break;
+        const unsigned long long keep_policy = l2_policy_evict_last();         // activations come back every pass
+        struct Item {
+            const __half* x;
+            int k_in, kb, uses, phase;
+            unsigned xs;
+        };
+        // iterator over this warp's blobs
+        int it_oi = -1, it_kb = 0, it_nkb = 0, it_kin = 0, it_phase = -1;
+        int fk0 = 0, fk1 = 0, lk0 = 0, lk1 = 0, n_mid = 0, two = 0;
+        unsigned xbase = 0;
+        const __half* it_x = nullptr;
+        auto advance = [&](Item& it) -> bool {
+            for (;;) {
+                if (it_kb < it_nkb) {
+                    int uses = n_mid + ((it_kb >= fk0 && it_kb < fk1) ? 1 : 0) + ((two && it_kb >= lk0 && it_kb < lk1) ? 1 : 0);
+                    it.x = it_x; it.k_in = it_kin; it.kb = it_kb; it.uses = uses * kBlobTiles; it.phase = it_phase;
+                    it.xs = xbase + (unsigned)it_kb;
+                    it_kb += kPrepWarps;
+                    return true;
+                }
+                xbase += (unsigned)it_nkb;
+                it_nkb = 0;
+                do { it_oi++; } while (it_oi < a.n_ops && range[it_oi].x == kRangeEmpty);
+                if (it_oi >= a.n_ops) return false;
+                prefetch_ops(ops, it_oi, a.n_ops, lane);
+                const GemvOp& op = ops[it_oi];
+                const StripOrder so(range[it_oi], op.n_kb);
+                it_nkb = op.n_kb; it_kin = op.k_in; it_phase = op.phase;
+                it_x = reinterpret_cast<const __half*>(op.x);
+                // blobs of x that this CTA's strips cover: the first and the last strip may be partial
+                int f0, f1, l0, l1;
+                so.chunks(so.rp_first, f0, f1);
+                so.chunks(so.rp_last, l0, l1);
+                fk0 = f0; fk1 = f1; lk0 = l0; lk1 = l1;
+                n_mid = so.n_strips > 2 ? so.n_strips - 2 : 0;
+                two = so.n_strips > 1;
+                it_kb = (int)(((unsigned)pw - xbase) % kPrepWarps);
+            }
+        };
+        // Is the phase that produces this op's activations complete?  (phases are opened in order)
+        auto phase_open = [&](int phase) -> bool { return phase <= 0 || (int)ctl[S::cPhaseKnown] >= phase; };
+        // Waits -- bounded -- until it is.  One warp of the CTA at a time polls the counters in global memory,
+        // always the earliest phase that is not known to be complete (a warp whose next blob belongs to a
+        // later phase must not keep a warp that still has to convert an earlier phase's activations from
+        // learning that it may go ahead); the others watch the word it updates in shared memory.
+        auto phase_wait = [&](int phase) -> bool {
+            int ok = 1;
+            if (lane == 0 && !phase_open(phase)) {
+                const unsigned long long t0 = global_ns();
+                unsigned it = 0;
+                for (;;) {
+                    if (phase_open(phase)) break;
+                    if (atomicCAS(const_cast<unsigned*>(&ctl[S::cPollLock]), 0u, 1u) == 0u) {
+                        while (ok && !phase_open(phase)) {
+                            const int p = (int)ctl[S::cPhaseKnown];                  // phases 0 .. p - 1 are complete
+                            const unsigned long long need = (unsigned long long)a.phase_total[p];
+                            while (ld_acquire_u64(a.phase_done + p) < need) {
+                                if ((++it & 31u) == 0u &&
+                                    (ctl[S::cAbort] || global_ns() - t0 > a.wait_ns || *reinterpret_cast<volatile int*>(a.status) != 0)) {
+                                    ok = 0; break;
+                                }
                             }
+                            if (ok) ctl[S::cPhaseKnown] = (unsigned)(p + 1);
                         }
-                    }
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) { stop = true; break; }
-                phase_known = op.phase - 1;
-            }
-            const __half* x = reinterpret_cast<const __half*>(op.x);
-            // this warp's blobs of the op: activation blob numbers congruent to pw; up to four per round
-            int kb = (int)((pw + kPrepWarps - (xseq % kPrepWarps)) % kPrepWarps);
-            while (kb < n_kb && !stop) {
-                uint4 raw[4][2];
-#pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    const int kq = kb + q * kPrepWarps;
-#pragma unroll
-                    for (int ss = 0; ss < 2; ss++) {
-                        raw[q][ss] = make_uint4(0u, 0u, 0u, 0u);
-                        const int k = kq * 512 + ss * 256 + lane * 8;
-                        if (kq < n_kb && k < op.k_in) raw[q][ss] = __ldcg(reinterpret_cast<const uint4*>(x + k));
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < 4; q++) {
-                    const int kq = kb + q * kPrepWarps;
-                    if (kq >= n_kb) break;
-                    const unsigned xs = xseq + (unsigned)kq;
-                    const int slot = (int)(xs % kXSlots);
-                    int uses = n_mid + ((kq >= fk0 && kq < fk1) ? 1 : 0);
-                    if (so.n_strips > 1) uses += (kq >= lk0 && kq < lk1) ? 1 : 0;
-                    uses *= kBlobTiles;
-                    int ok = 1;
-                    if (lane == 0 && !wait_smem([&] { return ctl[S::cXCnt + slot] == 0u; }, ctl, a.wait_ns)) {
-                        if (!ctl[S::cAbort]) raise_timeout(a, ctl);
-                        ok = 0;
-                    }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) { stop = true; break; }
-                    if (uses > 0) {
-                        uint8_t* xdig = smem + S::oXDig + slot * kXBlobDigitBytes;
-                        uint8_t* xgrp = smem + S::oXGrp + slot * kXBlobGroupBytes;
-                        convert_superstep(raw[q][0], xdig, xgrp, 0, lane);
-                        convert_superstep(raw[q][1], xdig, xgrp, 1, lane);
-                    }
-                    __threadfence_block();
-                    __syncwarp();
-                    if (lane == 0) {
-                        ctl[S::cXCnt + slot] = (unsigned)uses;
                         __threadfence_block();
-                        ctl[S::cXTag + slot] = xs + 1u;
+                        ctl[S::cPollLock] = 0u;
+                        break;
                     }
+                    __nanosleep(20);
+                    if ((++it & 63u) == 0u && (ctl[S::cAbort] || global_ns() - t0 > a.wait_ns)) { ok = 0; break; }
                 }
-                kb += 4 * kPrepWarps;
+                if (!ok && !ctl[S::cAbort]) raise_timeout(a, ctl);
             }
-            xseq += (unsigned)n_kb;
+            return __shfl_sync(0xffffffffu, ok, 0) != 0;
+        };
+        auto load = [&](const Item& it, uint4& r0, uint4& r1) {
+            r0 = r1 = make_uint4(0u, 0u, 0u, 0u);
+            const int k = it.kb * 512 + lane * 8;
+            if (it.uses > 0) {
+                if (k < it.k_in) r0 = ldg128_hint(it.x + k, keep_policy);
+                if (k + 256 < it.k_in) r1 = ldg128_hint(it.x + k + 256, keep_policy);
+            }
+        };
+        // Converts a blob into its slot and publishes it.  False: a wait ran out.
+        auto process = [&](const Item& it, uint4 r0, uint4 r1) -> bool {
+            const int slot = (int)(it.xs % kXSlots);
+            int ok = 1;
+            if (lane == 0 && !wait_smem([&] { return ctl[S::cXCnt + slot] == 0u; }, ctl, a.wait_ns)) {
+                if (!ctl[S::cAbort]) raise_timeout(a, ctl);
+                ok = 0;
+            }
+            if (!__shfl_sync(0xffffffffu, ok, 0)) return false;
+            if (it.uses > 0) {
+                uint8_t* xdig = smem + S::oXDig + slot * kXBlobDigitBytes;
+                uint8_t* xgrp = smem + S::oXGrp + slot * kXBlobGroupBytes;
+                convert_superstep(r0, xdig, xgrp, 0, lane);
+                convert_superstep(r1, xdig, xgrp, 1, lane);
+            }
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) {
+                ctl[S::cXCnt + slot] = (unsigned)it.uses;
+                __threadfence_block();
+                ctl[S::cXTag + slot] = it.xs + 1u;
+            }
+            return true;
+        };
+        Item A, B;
+        uint4 ra0, ra1, rb0, rb1;
+        bool va = advance(A);
+        if (va) {
+            if (!phase_wait(A.phase)) va = false;
+            else load(A, ra0, ra1);
+        }
+        while (va) {
+            const bool vb = advance(B);
+            bool issued = false;
+            if (vb && __shfl_sync(0xffffffffu, phase_open(B.phase) ? 1 : 0, 0)) { load(B, rb0, rb1); issued = true; }
+            if (!process(A, ra0, ra1)) break;
+            if (vb && !issued) {
+                if (!phase_wait(B.phase)) break;
+                load(B, rb0, rb1);
+            }
+            A = B; ra0 = rb0; ra1 = rb1; va = vb;
         }
     } else {
         // ================================================================== consumers
@@ -547,12 +638,15 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             __threadfence_block();
             bool live = true;
             if (finish) {
-                // lane = row of the strip; blob sums in blob order; blobs of other CTAs from their tagged words
-                const int n_kb = d.n_kb, kb_lo = d.kb_lo;
+                // lane = row of the strip; blob sums in blob order: this CTA's from shared memory, then the blobs
+                // of other CTAs from their tagged words
+                const int n_kb = d.n_kb, kb_hi = d.kb_hi;
                 float sum = 0.f;
-                if (kb_lo > 0) {
+                const float* ps = part + (sslot * kMaxKb) * 32 + lane;
+                for (int q = 0; q < kb_hi; q++) sum += ps[q * 32];
+                if (kb_hi < n_kb) {
                     const unsigned long long t0 = global_ns();
-                    for (int q = 0; q < kb_lo && live; q++) {
+                    for (int q = kb_hi; q < n_kb && live; q++) {
                         unsigned long long wv = ld_relaxed_u64(d.partial + q * 32 + lane);
                         unsigned it = 0;
                         while (!__all_sync(0xffffffffu, (unsigned)(wv >> 32) == a.epoch)) {
@@ -567,8 +661,6 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                     if (!live && lane == 0 && !ctl[S::cAbort]) raise_timeout(a, ctl);
                 }
                 if (live) {
-                    const float* ps = part + (sslot * kMaxKb) * 32 + lane;
-                    for (int q = kb_lo; q < n_kb; q++) sum += ps[q * 32];
                     const int row = d.row_base + lane;
                     if (row < d.n_out) reinterpret_cast<__half*>(d.y)[row] = __float2half_rn(sum);
                 }
@@ -635,7 +727,14 @@ unsigned next_epoch(unsigned& e)
 }  // namespace
 
 int gemv1_max_phases() { return kMaxPhasesDev; }
+int gemv1_max_ops() { return kMaxOpsDev; }
+uint2 gemv1_pack_range(const CtaWork& w, int n_chunks) { return pack_range(w, n_chunks); }
 int gemv1_max_k() { return kMaxKb * 512; }
+int gemv1_chunk_blobs(int blob_read_bytes)
+{
+    const int c = kStageBytes / blob_read_bytes;
+    return c > kBlobsMax ? kBlobsMax : (c < 1 ? 1 : c);
+}
 
 int launch_gemv1_single(Ctx* ctx, const GemvOp& op, cudaStream_t st)
 {
@@ -652,6 +751,9 @@ int launch_gemv1_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, 
     Args a{};
     a.table = reinterpret_cast<const GemvOp*>(table_dev);
     a.phase_total = reinterpret_cast<const int*>(table_dev + (size_t)hdr.n_ops * sizeof(GemvOp));
+    const size_t np = hdr.n_phases > 0 ? hdr.n_phases : 1;
+    a.ranges = reinterpret_cast<const uint2*>(
+        table_dev + (size_t)round_up((int64_t)((size_t)hdr.n_ops * sizeof(GemvOp) + np * sizeof(int)), 8));
     a.phase_done = reinterpret_cast<unsigned long long*>(ctx->ws);
     a.exit_count = reinterpret_cast<unsigned*>(ctx->ws + 8 * 4096);
     a.status = ctx->status_dev;

@@ -107,11 +107,15 @@ int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, 
 int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_bytes_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                 // batch 2..8
+struct CtaWork;
 int launch_gemv1_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                // batch 1
-// table_dev: [GemvOp x n_ops][int phase_total x max(n_phases,1)]
+// table_dev: [GemvOp x n_ops][int phase_total x max(n_phases,1)][uint2 strips x sm_count x n_ops]
 int launch_gemv1_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, cudaStream_t st);
 int gemv1_max_phases();
+int gemv1_max_ops();
 int gemv1_max_k();
+int gemv1_chunk_blobs(int blob_read_bytes);
+uint2 gemv1_pack_range(const CtaWork& w, int n_chunks);
 int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st);
 // table_dev: [GemvOp x n_ops][long long phase_total x max(n_phases,1)][int cta_units x sm_count]
 int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, int max_batch, cudaStream_t st);
@@ -119,8 +123,9 @@ int launch_gemv_stack(Ctx* ctx, const StackHeader& hdr, const char* table_dev, i
 void gemv_cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi);
 
 // ---- how a decode op is dealt to the CTAs of the persistent grid (shared by host and device code)
-// Units of an op (one unit = one K chunk of one 32-row strip) are numbered strip-major, u = rp * n_chunks + ch,
-// and dealt in contiguous blocks; the block boundaries rotate from op to op so that the remainders even out.
+// The pieces of an op (batch 1: the blobs of its 32-row strips; batch 2..8: K chunks of row pairs) are numbered
+// strip-major, u = rp * pieces_per_strip + i, and dealt in contiguous blocks; the block boundaries rotate from
+// op to op so that the remainders even out.
 FQ_HD void cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi)
 {
     const unsigned c = (unsigned)((cta + grid - rot) % grid);
@@ -131,17 +136,17 @@ FQ_HD void cta_range(int n_units, int rot, int cta, int grid, int& lo, int& hi)
 struct CtaWork {
     int lo, hi, rp_first, rp_last;
     FQ_HD bool any() const { return hi > lo; }
-    // chunks [c0, c1) of strip rp that belong to this CTA
+    // pieces [c0, c1) of strip rp that belong to this CTA
     FQ_HD void chunks(int n_chunks, int rp, int& c0, int& c1) const
     {
         c0 = rp == rp_first ? lo - rp * n_chunks : 0;
         c1 = rp == rp_last ? hi - rp * n_chunks : n_chunks;
     }
-    // strips that this CTA finishes (it owns their last chunk) and therefore writes to y
+    // strips that this CTA finishes (it owns their first piece) and therefore writes to y
     FQ_HD int finishing(int n_chunks) const
     {
         if (!any()) return 0;
-        return rp_last - rp_first + 1 - (hi - rp_last * n_chunks < n_chunks ? 1 : 0);
+        return rp_last - rp_first + 1 - (lo - rp_first * n_chunks > 0 ? 1 : 0);
     }
 };
 FQ_HD CtaWork cta_work(int n_units, int n_chunks, int rot, int cta, int grid)
