@@ -562,18 +562,28 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
                 int g1 = g0 + 1;
                 while (g1 < n_ops && (!phases_host || phases_host[g1] == phases_host[g0])) g1++;
                 unsigned long long total = 0;
-                for (int i = g0; i < g1; i++) total += (unsigned long long)ops[i].n_units * (unsigned)ops[i].blob_read;
+                long long strips = 0;
+                for (int i = g0; i < g1; i++) {
+                    total += (unsigned long long)ops[i].n_units * (unsigned)ops[i].blob_read;
+                    strips += ops[i].n_rp;
+                }
+                // A group with few strips per CTA is dealt in whole strips: such a phase is short, and what
+                // counts is that no CTA has to wait for a neighbour's share of a strip, not the last few
+                // per cent of balance.
+                const bool whole_strips = phases_host && strips < 2ll * grid;
                 const int rot = (int)((unsigned)group * 53u % (unsigned)grid);      // spreads the remainders
                 unsigned long long before = 0;
                 for (int i = g0; i < g1; i++) {
                     const unsigned long long sz = (unsigned)ops[i].blob_read;
                     const unsigned long long bytes = (unsigned long long)ops[i].n_units * sz;
+                    const unsigned long long strip_bytes = (unsigned long long)ops[i].n_kb * sz;
                     for (int c = 0; c < grid; c++) {
                         const unsigned long long cc = (unsigned)((c + grid - rot) % grid);
                         // blobs of this op whose first byte lies in [cut(cc), cut(cc + 1))
                         auto first_blob_at = [&](unsigned long long pos) -> long long {
                             if (pos <= before) return 0;
                             if (pos >= before + bytes) return ops[i].n_units;
+                            if (whole_strips) return (long long)((pos - before + strip_bytes - 1) / strip_bytes) * ops[i].n_kb;
                             return (long long)((pos - before + sz - 1) / sz);
                         };
                         CtaWork w;

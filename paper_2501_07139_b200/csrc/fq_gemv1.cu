@@ -15,9 +15,9 @@
 //   producer warp   : walks the op list, streams units into a ring of shared-memory stages with bulk
 //                     asynchronous copies (cp.async.bulk + mbarrier tx counts; it runs ahead across op and
 //                     phase boundaries because weights do not depend on activations) and deals the
-//                     (blob, 16-row tile) items of every unit round-robin into per-warp queues;
-//   consumer warps  : 16 warps = 8 K lanes x 2 row tiles.  An item is one tile of one blob: the arithmetic
-//                     of fq_gemv_core.cuh, then the 16 row sums go to the strip's slot in shared memory
+//                     blobs of every unit round-robin into per-warp queues;
+//   consumer warps  : 16 warps.  An item is one blob (32 rows x 512 columns): the arithmetic of
+//                     fq_gemv_core.cuh, then the 32 row sums go to the strip's slot in shared memory
 //                     (or to global memory for a strip finished elsewhere).  The warp that delivers a
 //                     strip's last item adds the blob sums up, writes y and counts the strip for its phase;
 //   x-prep warps    : convert the activations of every blob this CTA needs into 16-bit fixed point per
@@ -38,16 +38,16 @@ namespace fq {
 
 namespace {
 
-constexpr int kCW = 16;                                // consumer warps: K lane = warp >> 1, row tile = warp & 1
-constexpr int kKLanes = kCW / kBlobTiles;
+constexpr int kCW = 16;                                // consumer warps; consecutive blobs go to consecutive warps
+constexpr int kKLanes = kCW;
 constexpr int kProducerWarp = kCW;
 constexpr int kPrepWarp = kCW + 1;                     // first activation pre-processing warp
-constexpr int kPrepWarps = 8;
+constexpr int kPrepWarps = 7;                          // 24 warps in all: 80 registers per thread
 constexpr int kThreads = (kCW + 1 + kPrepWarps) * 32;
 constexpr int kStageBytes = 34816;                     // one unit: 4 x 4-bit blobs or 2 x 8-bit blobs
 constexpr int kBlobsMax = 6;                           // blobs per unit, at most (< kKLanes: a warp gets at most one item of a unit)
-constexpr int kXSlots = 32;                            // activation blobs resident in shared memory
-constexpr int kStripSlots = 4;                         // strips whose items are in flight
+constexpr int kXSlots = 28;                            // activation blobs resident in shared memory
+constexpr int kStripSlots = 5;                         // strips whose items are in flight
 constexpr int kMaxKb = 28;                             // blobs per strip, at most (k_in <= 14336)
 constexpr int kQD = 8;                                 // entries per consumer queue
 constexpr int kMaxPhasesDev = 1024;
@@ -321,7 +321,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         const uint32_t sdesc_a = sbase + S::oStrip;
         const unsigned long long stream_policy = l2_policy_evict_first();      // weights are read once per pass
         const uint32_t my_queue = sbase + S::oQueue + (uint32_t)(lane & (kCW - 1)) * kQD * 16u;
-        const int my_klane = (lane >> 1) & (kKLanes - 1), my_tile = lane & 1;
+        const int my_klane = lane & (kKLanes - 1);
         // The descriptor of the next op travels while the units of the current one are issued.
         struct OpRegs {
             const uint8_t* store;
@@ -370,7 +370,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                     if (lane == 0) d = make_uint4((uint32_t)(uintptr_t)y, (uint32_t)((uintptr_t)y >> 32), (uint32_t)(uintptr_t)sp,
                                                   (uint32_t)((uintptr_t)sp >> 32));
                     else if (lane == 1) d = make_uint4((uint32_t)n_out, (uint32_t)(rp * (kBlobTiles * kTileRows)), (uint32_t)n_kb, (uint32_t)kb_lo);
-                    else d = make_uint4((uint32_t)kb_hi, c0 == 0 ? 1u : 0u, (uint32_t)phase, (uint32_t)((kb_hi - kb_lo) * kBlobTiles));
+                    else d = make_uint4((uint32_t)kb_hi, c0 == 0 ? 1u : 0u, (uint32_t)phase, (uint32_t)(kb_hi - kb_lo));
                     if (lane < 3) sts128(sdesc_a + (uint32_t)sslot * 64u + (uint32_t)lane * 16u, d);
                     if (lane == 0) ctl[S::cStripBusy + sslot] = 1u;
                     __threadfence_block();                           // the descriptor before any item that refers to it
@@ -390,13 +390,13 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                         if (ok) {
                             mbar_expect_tx(full, (uint32_t)nb * blob_read);
                             if (contiguous) bulk_g2s_hint(stage_base, src, (uint32_t)nb * blob_read, full, stream_policy);
-                            mbar_arrive_n(empty, (uint32_t)(kCW - nb * kBlobTiles));   // for the warps without an item in this unit
+                            mbar_arrive_n(empty, (uint32_t)(kCW - nb));   // for the warps without an item in this unit
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) { stop = true; break; }
                     if (!contiguous && lane < nb) bulk_g2s_hint(stage_base + lane * blob_read, src + lane * blob_stride, blob_read, full, stream_policy);
-                    // the items of this unit: blob b goes to K lane (rr + b) mod 8, its two tiles to that lane's two warps
+                    // the items of this unit: blob b goes to consumer warp (rr + b) mod 16
                     const int b = (int)((unsigned)my_klane - rr) & (kKLanes - 1);
                     if (lane < kCW && b < nb) {
                         const unsigned xs = xseq + (unsigned)(kb + b);
@@ -408,7 +408,6 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                         sts128(my_queue + (qn % kQD) * 16u, e);
                         qn++;
                     }
-                    (void)my_tile;
                     rr += (unsigned)nb;
                     src += (long long)nb * blob_stride;
                     if (++stage == S::kStages) { stage = 0; wraps++; }
@@ -418,7 +417,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         }
         // the end marker of every queue
         if (lane < kCW) {
-            // (the queue slot is free: a warp gets one entry per kKLanes blobs, so the entry that used the slot
+            // (the queue slot is free: a warp gets one entry per kCW blobs, so the entry that used the slot
             // kQD entries ago belongs to a unit whose stage has been refilled since, i.e. it was consumed)
             sts128(my_queue + (qn % kQD) * 16u, make_uint4(0u, kItemEnd, 0u, qn + 1u));
         }
@@ -451,7 +450,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             for (;;) {
                 if (it_kb < it_nkb) {
                     int uses = n_mid + ((it_kb >= fk0 && it_kb < fk1) ? 1 : 0) + ((two && it_kb >= lk0 && it_kb < lk1) ? 1 : 0);
-                    it.x = it_x; it.k_in = it_kin; it.kb = it_kb; it.uses = uses * kBlobTiles; it.phase = it_phase;
+                    it.x = it_x; it.k_in = it_kin; it.kb = it_kb; it.uses = uses; it.phase = it_phase;
                     it.xs = xbase + (unsigned)it_kb;
                     it_kb += kPrepWarps;
                     return true;
@@ -472,7 +471,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                 fk0 = f0; fk1 = f1; lk0 = l0; lk1 = l1;
                 n_mid = so.n_strips > 2 ? so.n_strips - 2 : 0;
                 two = so.n_strips > 1;
-                it_kb = (int)(((unsigned)pw - xbase) % kPrepWarps);
+                it_kb = (int)(((unsigned)pw + kPrepWarps - xbase % kPrepWarps) % kPrepWarps);
             }
         };
         // Is the phase that produces this op's activations complete?  (phases are opened in order)
@@ -563,7 +562,6 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         }
     } else {
         // ================================================================== consumers
-        const int tile = warp & 1;
         const int g = lane >> 2, c = lane & 3;
         const uint32_t queue = sbase + S::oQueue + (uint32_t)warp * kQD * 16u;
         const StripDesc* sdesc = reinterpret_cast<const StripDesc*>(smem + S::oStrip);
@@ -606,25 +604,28 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
 #pragma unroll
             for (int jc = 0; jc < 4; jc++)
                 xd[jc] = (g >> 1) == jc ? xdig + x_digit_off(0, jc, g & 1, c) : sbase + S::oZero + c * 16;
-            float tot[2] = {0.f, 0.f};
-            blob_tile_dispatch(variant, e.x, tile, xd, sbase + S::oXGrp + (uint32_t)xslot * kXBlobGroupBytes, lane, tot);
+            float tot[kBlobTiles][2] = {{0.f, 0.f}, {0.f, 0.f}};
+            blob_dispatch(variant, e.x, xd, sbase + S::oXGrp + (uint32_t)xslot * kXBlobGroupBytes, lane, tot);
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(bars + 128 + 8 * stage);                         // the stage may be refilled
                 atomicSub(const_cast<unsigned*>(&ctl[S::cXCnt + xslot]), 1u);   // one item fewer needs the activation blob
             }
-            // ---- the 16 row sums of the item: add up the step classes held by the quad
+            // ---- the 32 row sums of the item: add up the step classes held by the quad; lane c of the quad
+            //      then keeps the sum of row 16 (c >> 1) + g + 8 (c & 1)
 #pragma unroll
-            for (int r = 0; r < 2; r++) {
-                tot[r] += __shfl_xor_sync(0xffffffffu, tot[r], 1);
-                tot[r] += __shfl_xor_sync(0xffffffffu, tot[r], 2);
-            }
+            for (int tl = 0; tl < kBlobTiles; tl++)
+#pragma unroll
+                for (int r = 0; r < 2; r++) {
+                    tot[tl][r] += __shfl_xor_sync(0xffffffffu, tot[tl][r], 1);
+                    tot[tl][r] += __shfl_xor_sync(0xffffffffu, tot[tl][r], 2);
+                }
             const StripDesc& d = sdesc[sslot];
             const int finish = d.finish, expect = d.expect;                  // (read before this item is counted)
             unsigned long long* const dpart = d.partial;
-            if (c < 2) {                                                     // lane c of the quad stores row g + 8 c
-                const float v = c == 0 ? tot[0] : tot[1];
-                const int lr = tile * kTileRows + g + 8 * c;
+            {
+                const float v = c == 0 ? tot[0][0] : c == 1 ? tot[0][1] : c == 2 ? tot[1][0] : tot[1][1];
+                const int lr = (c >> 1) * kTileRows + g + 8 * (c & 1);
                 if (finish) part[(sslot * kMaxKb + kb) * 32 + lr] = v;
                 else st_relaxed_u64(dpart + kb * 32 + lr, tag | __float_as_uint(v));   // finished elsewhere
             }

@@ -1,5 +1,5 @@
-// Decode arithmetic of one work item: one 16-row tile of one blob (512 columns = two supersteps
-// of 256), batch 1.  Included by the decode kernel only.
+// Decode arithmetic of one work item: one blob (two 16-row tiles x 512 columns = two supersteps of 256),
+// batch 1.  Included by the decode kernel only.
 //
 // Stored words become A operands of the 8-bit mma.m16n8k32 with ONE AND each (a word holds 8/F
 // registers on top of each other, see fq_layout.cuh); the activations are 16-bit fixed point per
@@ -133,70 +133,72 @@ __device__ __forceinline__ void field_step(uint32_t fa, const uint4 (&bx)[4], in
     }
 }
 
-// The fields of one superstep, unrolled at compile time from the variant's field list.
-//   ST : superstep * 2 + tile parity is not known at compile time: the tile offset is passed in `fbase`
-template <int VARIANT, int FI, int PREFIX, int SS>
+// The fields of one (superstep, tile), unrolled at compile time from the variant's field list.
+template <int VARIANT, int FI, int PREFIX, int SS, int TILE>
 struct FieldLoop {
-    static __device__ __forceinline__ void run(uint32_t fbase, int tile, const uint4 (&bx)[4], int c, int m1, int (&v)[2][2])
+    static __device__ __forceinline__ void run(uint32_t fbase, const uint4 (&bx)[4], int c, int m1, int (&v)[2][2])
     {
         constexpr FieldList FL = variant_fields(VARIANT);
         if constexpr (FI < FL.n) {
             constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
-            // field array of width F after fields adding up to PREFIX bits; tile (SS, tile) of it
-            constexpr int off = kBlobSteps * kBlobTiles * 512 * PREFIX + SS * kBlobTiles * (F * 512);
-            field_step<F, SHIFT, FI == 0, off>(fbase + tile * (F * 512), bx, c, m1, v);
-            FieldLoop<VARIANT, FI + 1, PREFIX + F, SS>::run(fbase, tile, bx, c, m1, v);
+            // field array of width F after fields adding up to PREFIX bits; tile (SS, TILE) of it
+            constexpr int off = kBlobSteps * kBlobTiles * 512 * PREFIX + (SS * kBlobTiles + TILE) * (F * 512);
+            field_step<F, SHIFT, FI == 0, off>(fbase, bx, c, m1, v);
+            FieldLoop<VARIANT, FI + 1, PREFIX + F, SS, TILE>::run(fbase, bx, c, m1, v);
         }
     }
 };
 
-// One blob x one tile: tot[r] += dequantised dot products of rows g + 8 r (this lane's step class only;
-// the four lanes of a quad add up to the row sums).
+// One blob (32 rows x 512 columns): tot[tile][r] += dequantised dot products of rows 16 tile + g + 8 r (this
+// lane's step class only; the four lanes of a quad add up to the row sums).  Both row tiles share the B
+// registers and the group sums of the activations.
 //   blob : shared address of the blob          xd : this lane's B source per step class (digits or zeros)
 //   xg   : shared address of the blob's group sums / scales
 template <int VARIANT>
-__device__ __forceinline__ void blob_tile(uint32_t blob, int tile, const uint32_t (&xd)[4], uint32_t xg, int lane,
-                                          float (&tot)[2])
+__device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane, float (&tot)[kBlobTiles][2])
 {
     // a nested child reads the parent's top bits; the dropped bits are filled with their mid-point, which
     // is the same as lowering every zero point by that amount
     constexpr int kAdjust = (VARIANT >= 7 && VARIANT < 13) ? 1 << (7 - (VARIANT - 5)) : 0;
     const int g = lane >> 2, c = lane & 3;
     const uint32_t fbase = blob + kBlobMetaBytes + lane * 16;
-    const uint32_t mbase = blob + tile * 128 + g * 16;
+    const uint32_t mbase = blob + g * 16;
     const int m1 = opaque_minus_one();
     const int czero = c == 0 ? m1 : 0;                         // only the class-0 lane of a quad subtracts the zero-point term
     static_for<0, kBlobSteps>([&](auto SSI) {
         constexpr int ss = decltype(SSI)::value;
         uint4 bx[4];
         static_for<0, 4>([&](auto JC) { bx[decltype(JC)::value] = lds128<ss * 512>(xd[decltype(JC)::value]); });
-        const uint4 mw = lds128<ss * (kBlobTiles * 128)>(mbase);        // (grp 0: row g, g + 8), (grp 1: row g, g + 8)
         const uint2 xs2 = lds64<ss * 8>(xg), sc2 = lds64<16 + ss * 8>(xg);
-        int v[2][2];
-        FieldLoop<VARIANT, 0, 0, ss>::run(fbase, tile, bx, c, m1, v);
-        // group epilogue: y += s * 2^-e * (v - (z - adjust) * sum x_int)
         const int nx[2] = {(int)xs2.x * czero, (int)xs2.y * czero};
         const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
-        const uint32_t mm[2][2] = {{mw.x, mw.y}, {mw.z, mw.w}};
+        static_for<0, kBlobTiles>([&](auto TLI) {
+            constexpr int tile = decltype(TLI)::value;
+            const uint4 mw = lds128<(ss * kBlobTiles + tile) * 128>(mbase);   // (grp 0: row g, g + 8), (grp 1: row g, g + 8)
+            int v[2][2];
+            FieldLoop<VARIANT, 0, 0, ss, tile>::run(fbase, bx, c, m1, v);
+            // group epilogue: y += s * 2^-e * (v - (z - adjust) * sum x_int)
+            const uint32_t mm[2][2] = {{mw.x, mw.y}, {mw.z, mw.w}};
 #pragma unroll
-        for (int grp = 0; grp < 2; grp++) {
-            const int base = kAdjust ? -kAdjust * nx[grp] : 0;
+            for (int grp = 0; grp < 2; grp++) {
+                const int base = kAdjust ? -kAdjust * nx[grp] : 0;
 #pragma unroll
-            for (int r = 0; r < 2; r++) {
-                const uint32_t m = mm[grp][r];
-                const float s = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
-                const int t = v[grp][r] + (int)__umulhi(m, 65536u) * nx[grp] + base;
-                tot[r] = fmaf((float)t, s * sc[grp], tot[r]);
+                for (int r = 0; r < 2; r++) {
+                    const uint32_t m = mm[grp][r];
+                    const float s = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
+                    const int t = v[grp][r] + (int)__umulhi(m, 65536u) * nx[grp] + base;
+                    tot[tile][r] = fmaf((float)t, s * sc[grp], tot[tile][r]);
+                }
             }
-        }
+        });
     });
 }
 
 // Selects the specialised loop of a variant (variant_index in fq_layout.cuh).
-__device__ __forceinline__ void blob_tile_dispatch(int variant, uint32_t blob, int tile, const uint32_t (&xd)[4], uint32_t xg,
-                                                   int lane, float (&tot)[2])
+__device__ __forceinline__ void blob_dispatch(int variant, uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane,
+                                              float (&tot)[kBlobTiles][2])
 {
-#define FQ_VARIANT_CASE(V) case V: blob_tile<V>(blob, tile, xd, xg, lane, tot); break;
+#define FQ_VARIANT_CASE(V) case V: blob_compute<V>(blob, xd, xg, lane, tot); break;
     switch (variant) {
         FQ_VARIANT_CASE(0) FQ_VARIANT_CASE(1) FQ_VARIANT_CASE(2) FQ_VARIANT_CASE(3) FQ_VARIANT_CASE(4)
         FQ_VARIANT_CASE(5) FQ_VARIANT_CASE(6) FQ_VARIANT_CASE(7) FQ_VARIANT_CASE(8) FQ_VARIANT_CASE(9)
