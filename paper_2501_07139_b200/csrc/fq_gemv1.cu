@@ -52,7 +52,6 @@ constexpr int kMaxKb = 28;                             // blobs per strip, at mo
 constexpr int kQD = 8;                                 // entries per consumer queue
 constexpr int kMaxPhasesDev = 1024;
 constexpr int kMaxOpsDev = 512;                        // ops of one launch (their per-CTA ranges sit in shared memory)
-static_assert(kXSlots % kPrepWarps == 0, "an activation slot is always filled by the same warp");
 
 // What the producer tells a consumer warp about one item (one 16-byte store, one 16-byte load).
 //   w0 blob shared address   w1 packed fields (below)   w2 activation blob number + 1   w3 sequence tag
@@ -77,7 +76,7 @@ struct StripDesc {
 static_assert(sizeof(StripDesc) == 64, "descriptor layout");
 
 struct Smem {
-    static constexpr int kFixed = kXSlots * (kXBlobDigitBytes + kXBlobGroupBytes) + 1024 + kStripSlots * kMaxKb * 128 +
+    static constexpr int kFixed = kXSlots * (kXBlobDigitBytes + kXBlobGroupBytes + 8) + 1024 + kStripSlots * kMaxKb * 128 +
                                   kCW * kQD * 16 + kStripSlots * 64 + kMaxPhasesDev + kMaxOpsDev * 8 + 1024;
     static constexpr int kStages = (232448 - kFixed) / kStageBytes;
     static constexpr int oStages = 0;
@@ -89,8 +88,8 @@ struct Smem {
     static constexpr int oStrip = oQueue + kCW * kQD * 16;                   // StripDesc [strip slot]
     static constexpr int oRange = oStrip + kStripSlots * 64;                 // uint2 [op]: this CTA's strips of every op
     static constexpr int oFinTot = oRange + kMaxOpsDev * 8;                  // u8 [phase]: strips this CTA finishes
-    static constexpr int oBars = oFinTot + kMaxPhasesDev;                    // full[S], empty[S]
-    static constexpr int oCtl = oBars + 2 * 16 * 8;
+    static constexpr int oBars = oFinTot + kMaxPhasesDev;                    // full[S], empty[S], then one per activation slot
+    static constexpr int oCtl = oBars + 2 * 16 * 8 + kXSlots * 8;
     // control words (u32 each)
     static constexpr int cXTag = 0;                                          // [kXSlots] activation blob number + 1 held
     static constexpr int cXCnt = cXTag + kXSlots;                            // [kXSlots] items that still need the slot
@@ -203,60 +202,82 @@ __device__ __forceinline__ bool wait_mbar(uint32_t bar, uint32_t parity, volatil
 }
 
 // ------------------------------------------------------------------------------- activation pre-processing
-// One superstep (256 columns, 8 per lane) of fp16 activations -> fixed point per group of 128 columns:
-// x_int = rint(x * 2^(13 - E)) with 2^E <= max|x| < 2^(E+1), stored as two signed byte digits in
+// One blob (two supersteps of 256 columns, 8 per lane each) of fp16 activations -> fixed point per group of
+// 128 columns: x_int = rint(x * 2^(13 - E)) with 2^E <= max|x| < 2^(E+1), stored as two signed byte digits in
 // B-fragment order, plus per group the integer sum and the factor 2^(E - 13).  A group that holds an
-// infinity or a NaN gets the factor NaN, so that every row sum that touches it comes out NaN.
-__device__ __forceinline__ void convert_superstep(uint4 raw, uint8_t* xdig, uint8_t* xgrp, int ss, int lane)
+// infinity or a NaN gets the factor NaN, so that every row sum that touches it comes out NaN.  The two
+// supersteps are independent chains of shuffles and conversions: written side by side so that their
+// latencies overlap.
+__device__ __forceinline__ void convert_blob(const uint4 (&raw)[2], uint8_t* xdig, uint8_t* xgrp, int lane)
 {
-    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-    float f[8];
-    bool bad = false;
+    float f[2][8], amax[2];
+    bool bad[2];
 #pragma unroll
-    for (int i = 0; i < 4; i++) {
-        const float2 t2 = __half22float2(h2[i]);
-        f[2 * i] = t2.x; f[2 * i + 1] = t2.y;
+    for (int ss = 0; ss < 2; ss++) {
+        const __half2* h2 = reinterpret_cast<const __half2*>(&raw[ss]);
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            const float2 t2 = __half22float2(h2[i]);
+            f[ss][2 * i] = t2.x; f[ss][2 * i + 1] = t2.y;
+        }
+        float m01 = fmaxf(fabsf(f[ss][0]), fabsf(f[ss][1])), m23 = fmaxf(fabsf(f[ss][2]), fabsf(f[ss][3]));
+        float m45 = fmaxf(fabsf(f[ss][4]), fabsf(f[ss][5])), m67 = fmaxf(fabsf(f[ss][6]), fabsf(f[ss][7]));
+        amax[ss] = fmaxf(fmaxf(m01, m23), fmaxf(m45, m67));
+        // an infinity or a NaN: |x| <= 65504 fails for both (fmaxf drops a NaN, so test the elements)
+        bool ok = true;
+#pragma unroll
+        for (int i = 0; i < 8; i++) ok = ok && (fabsf(f[ss][i]) <= 65504.f);
+        bad[ss] = !ok;
     }
-    float amax = 0.f;
 #pragma unroll
-    for (int i = 0; i < 8; i++) {
-        amax = fmaxf(amax, fabsf(f[i]));
-        bad = bad || !(fabsf(f[i]) <= 65504.f);                 // infinity or NaN
+    for (int o = 8; o > 0; o >>= 1) {
+        amax[0] = fmaxf(amax[0], __shfl_xor_sync(0xffffffffu, amax[0], o));
+        amax[1] = fmaxf(amax[1], __shfl_xor_sync(0xffffffffu, amax[1], o));
+    }
+    const unsigned badmask0 = __ballot_sync(0xffffffffu, bad[0]), badmask1 = __ballot_sync(0xffffffffu, bad[1]);
+    bad[0] = ((badmask0 >> (lane & 16)) & 0xffffu) != 0u;       // anywhere in this lane's group of 16 lanes
+    bad[1] = ((badmask1 >> (lane & 16)) & 0xffffu) != 0u;
+    int xi[2][8], sum[2];
+    float back[2];
+#pragma unroll
+    for (int ss = 0; ss < 2; ss++) {
+        const int eb = (__float_as_int(amax[ss]) >> 23) & 0xff;  // biased exponent of the group maximum
+        const bool fin = amax[ss] > 0.f && !bad[ss];
+        const float mult = fin ? __int_as_float((267 - eb) << 23) : 0.f;
+        back[ss] = bad[ss] ? __int_as_float(0x7fc00000) : (fin ? __int_as_float((eb - 13) << 23) : 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; i++) xi[ss][i] = bad[ss] ? 0 : __float2int_rn(f[ss][i] * mult);
+        sum[ss] = ((xi[ss][0] + xi[ss][1]) + (xi[ss][2] + xi[ss][3])) + ((xi[ss][4] + xi[ss][5]) + (xi[ss][6] + xi[ss][7]));
     }
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const unsigned badmask = __ballot_sync(0xffffffffu, bad);
-    bad = ((badmask >> (lane & 16)) & 0xffffu) != 0u;           // anywhere in this lane's group of 16 lanes
-    const int eb = (__float_as_int(amax) >> 23) & 0xff;         // biased exponent of the group maximum
-    const bool fin = amax > 0.f && !bad;
-    const float mult = fin ? __int_as_float((267 - eb) << 23) : 0.f;
-    const float back = bad ? __int_as_float(0x7fc00000) : (fin ? __int_as_float((eb - 13) << 23) : 0.f);
-    int xi[8], sum = 0;
-#pragma unroll
-    for (int i = 0; i < 8; i++) { xi[i] = bad ? 0 : __float2int_rn(f[i] * mult); sum += xi[i]; }
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    // signed digits base 256 of four values at a time: low byte as is, high byte + carry
-    uint32_t lo4[2], hi4[2];
-#pragma unroll
-    for (int r = 0; r < 2; r++) {
-        const uint32_t p01 = __byte_perm((uint32_t)xi[4 * r + 0], (uint32_t)xi[4 * r + 1], 0x5410);
-        const uint32_t p23 = __byte_perm((uint32_t)xi[4 * r + 2], (uint32_t)xi[4 * r + 3], 0x5410);
-        const uint32_t h01 = (((p01 >> 8) & 0x00ff00ffu) + ((p01 >> 7) & 0x00010001u)) & 0x00ff00ffu;
-        const uint32_t h23 = (((p23 >> 8) & 0x00ff00ffu) + ((p23 >> 7) & 0x00010001u)) & 0x00ff00ffu;
-        lo4[r] = __byte_perm(p01, p23, 0x6420);
-        hi4[r] = __byte_perm(h01, h23, 0x6420);
+    for (int o = 8; o > 0; o >>= 1) {
+        sum[0] += __shfl_xor_sync(0xffffffffu, sum[0], o);
+        sum[1] += __shfl_xor_sync(0xffffffffu, sum[1], o);
     }
-    // lane l holds columns 8l .. 8l+7: k32 step j = l >> 2, half (l >> 1) & 1, column blocks c0 and c0 + 1
+    // lane l holds columns 8l .. 8l+7 of a superstep: k32 step j = l >> 2, half (l >> 1) & 1, column blocks c0, c0 + 1
     const int j = lane >> 2, half = (lane >> 1) & 1, c0 = 2 * (lane & 1);
-    uint8_t* cell = xdig + x_digit_off(ss, j & 3, 0, c0) + (2 * (j >> 2) + half) * 4;
-    *reinterpret_cast<uint32_t*>(cell) = lo4[0];
-    *reinterpret_cast<uint32_t*>(cell + 16) = lo4[1];
-    *reinterpret_cast<uint32_t*>(cell + 64) = hi4[0];
-    *reinterpret_cast<uint32_t*>(cell + 64 + 16) = hi4[1];
-    if ((lane & 15) == 0) {
-        reinterpret_cast<int*>(xgrp)[ss * 2 + (lane >> 4)] = sum;
-        reinterpret_cast<float*>(xgrp + 16)[ss * 2 + (lane >> 4)] = back;
+#pragma unroll
+    for (int ss = 0; ss < 2; ss++) {
+        // signed digits base 256 of four values at a time: low byte as is, high byte + carry
+        uint32_t lo4[2], hi4[2];
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+            const uint32_t p01 = __byte_perm((uint32_t)xi[ss][4 * r + 0], (uint32_t)xi[ss][4 * r + 1], 0x5410);
+            const uint32_t p23 = __byte_perm((uint32_t)xi[ss][4 * r + 2], (uint32_t)xi[ss][4 * r + 3], 0x5410);
+            const uint32_t h01 = (((p01 >> 8) & 0x00ff00ffu) + ((p01 >> 7) & 0x00010001u)) & 0x00ff00ffu;
+            const uint32_t h23 = (((p23 >> 8) & 0x00ff00ffu) + ((p23 >> 7) & 0x00010001u)) & 0x00ff00ffu;
+            lo4[r] = __byte_perm(p01, p23, 0x6420);
+            hi4[r] = __byte_perm(h01, h23, 0x6420);
+        }
+        uint8_t* cell = xdig + x_digit_off(ss, j & 3, 0, c0) + (2 * (j >> 2) + half) * 4;
+        *reinterpret_cast<uint32_t*>(cell) = lo4[0];
+        *reinterpret_cast<uint32_t*>(cell + 16) = lo4[1];
+        *reinterpret_cast<uint32_t*>(cell + 64) = hi4[0];
+        *reinterpret_cast<uint32_t*>(cell + 64 + 16) = hi4[1];
+        if ((lane & 15) == 0) {
+            reinterpret_cast<int*>(xgrp)[ss * 2 + (lane >> 4)] = sum[ss];
+            reinterpret_cast<float*>(xgrp + 16)[ss * 2 + (lane >> 4)] = back[ss];
+        }
     }
 }
 
@@ -280,6 +301,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             mbar_init(bars + 8 * s, 1);
             mbar_init(bars + 128 + 8 * s, kCW);
         }
+        for (int s = 0; s < kXSlots; s++) mbar_init(bars + 256 + 8 * s, 1);   // completes once per publication of the slot
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -522,7 +544,9 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         auto process = [&](const Item& it, uint4 r0, uint4 r1) -> bool {
             const int slot = (int)(it.xs % kXSlots);
             int ok = 1;
-            if (lane == 0 && !wait_smem([&] { return ctl[S::cXCnt + slot] == 0u; }, ctl, a.wait_ns)) {
+            // the slot is free when the blob it held before has been published and every item that needed it is done
+            const unsigned prev_tag = it.xs >= (unsigned)kXSlots ? it.xs - (unsigned)kXSlots + 1u : 0u;
+            if (lane == 0 && !wait_smem([&] { return ctl[S::cXTag + slot] == prev_tag && ctl[S::cXCnt + slot] == 0u; }, ctl, a.wait_ns)) {
                 if (!ctl[S::cAbort]) raise_timeout(a, ctl);
                 ok = 0;
             }
@@ -530,15 +554,16 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             if (it.uses > 0) {
                 uint8_t* xdig = smem + S::oXDig + slot * kXBlobDigitBytes;
                 uint8_t* xgrp = smem + S::oXGrp + slot * kXBlobGroupBytes;
-                convert_superstep(r0, xdig, xgrp, 0, lane);
-                convert_superstep(r1, xdig, xgrp, 1, lane);
+                const uint4 raw[2] = {r0, r1};
+                convert_blob(raw, xdig, xgrp, lane);
             }
             __threadfence_block();
             __syncwarp();
             if (lane == 0) {
                 ctl[S::cXCnt + slot] = (unsigned)it.uses;
-                __threadfence_block();
                 ctl[S::cXTag + slot] = it.xs + 1u;
+                __threadfence_block();
+                mbar_arrive(bars + 256 + 8 * slot);                        // wakes the consumers that sleep on this slot
             }
             return true;
         };
@@ -593,7 +618,9 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             const int kb = (int)((e.y >> 10) & 31u), sslot = (int)((e.y >> 15) & 7u), variant = (int)((e.y >> 18) & 15u);
             // ---- its weights and its activations
             bool ok = wait_mbar(bars + 8 * stage, (uint32_t)parity, ctl, a.wait_ns);
-            if (ok) ok = wait_smem([&] { return ctl[S::cXTag + xslot] == e.z; }, ctl, a.wait_ns);
+            // (a hardware wake-up: at the start of a dependency phase every consumer sleeps here and must not
+            // take issue slots from the pre-processing warps; the slot's barrier completes once per publication)
+            if (ok) ok = wait_mbar(bars + 256 + 8 * xslot, ((e.z - 1u) / kXSlots) & 1u, ctl, a.wait_ns);
             if (!__all_sync(0xffffffffu, ok)) {
                 if (lane == 0 && !ctl[S::cAbort]) raise_timeout(a, ctl);
                 break;
@@ -644,20 +671,33 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                 const int n_kb = d.n_kb, kb_hi = d.kb_hi;
                 float sum = 0.f;
                 const float* ps = part + (sslot * kMaxKb) * 32 + lane;
-                for (int q = 0; q < kb_hi; q++) sum += ps[q * 32];
+                for (int q0 = 0; q0 < kb_hi; q0 += 8) {                      // eight loads in flight, added in blob order
+                    float pv[8];
+#pragma unroll
+                    for (int i = 0; i < 8; i++) pv[i] = q0 + i < kb_hi ? ps[(q0 + i) * 32] : 0.f;
+#pragma unroll
+                    for (int i = 0; i < 8; i++) if (q0 + i < kb_hi) sum += pv[i];
+                }
                 if (kb_hi < n_kb) {
+                    // eight words in flight per round trip; a round whose words are not all there is repeated
                     const unsigned long long t0 = global_ns();
-                    for (int q = kb_hi; q < n_kb && live; q++) {
-                        unsigned long long wv = ld_relaxed_u64(d.partial + q * 32 + lane);
-                        unsigned it = 0;
-                        while (!__all_sync(0xffffffffu, (unsigned)(wv >> 32) == a.epoch)) {
+                    unsigned it = 0;
+                    for (int q0 = kb_hi; q0 < n_kb && live; q0 += 8) {
+                        unsigned long long wv[8];
+                        for (;;) {
+                            bool all = true;
+#pragma unroll
+                            for (int i = 0; i < 8; i++) wv[i] = q0 + i < n_kb ? ld_relaxed_u64(d.partial + (q0 + i) * 32 + lane) : tag;
+#pragma unroll
+                            for (int i = 0; i < 8; i++) all = all && (unsigned)(wv[i] >> 32) == a.epoch;
+                            if (__all_sync(0xffffffffu, all)) break;
                             __nanosleep(64);
                             int giveup = 0;
                             if (lane == 0 && (++it & 15u) == 0u && (ctl[S::cAbort] || global_ns() - t0 > a.wait_ns)) giveup = 1;
                             if (__shfl_sync(0xffffffffu, giveup, 0)) { live = false; break; }
-                            wv = ld_relaxed_u64(d.partial + q * 32 + lane);
                         }
-                        sum += __uint_as_float((unsigned)wv);
+#pragma unroll
+                        for (int i = 0; i < 8; i++) if (q0 + i < n_kb) sum += __uint_as_float((unsigned)wv[i]);
                     }
                     if (!live && lane == 0 && !ctl[S::cAbort]) raise_timeout(a, ctl);
                 }
