@@ -164,28 +164,32 @@ int fq_sqdiff(const uint16_t* a_bf16_dev, const uint16_t* b_bf16_dev, size_t n, 
 
 /* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.
- * Enqueues kernels on `stream`; does not synchronise. */
+ *   k_in <= 14336 (the activations of one 32-row strip stay in shared memory); FQ_ERR_SHAPE otherwise.
+ * Enqueues one kernel on `stream`; neither allocates (the scratch was reserved by fq_pack_layer) nor
+ * synchronises.  An activation group that holds an infinity or a NaN makes every output NaN. */
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
 
 /* Same result as fq_gemv, for callers that must not allocate device memory.  (The paper has no
- * counterpart; this is a deployment convenience.)  fq_gemv may grow the context's workspace
- * with cudaMalloc when a layer needs more split-K scratch than any earlier call did.  That is
+ * counterpart; this is a deployment convenience.)  fq_gemv takes its scratch from the context's
+ * workspace, device memory that fq_create / fq_pack_layer obtained with cudaMalloc.  That is
  * not acceptable for callers such as a real-time serving loop with a fixed memory budget, code
  * running while another library owns the allocator, or a host thread that must never block on
- * the device-wide synchronisation an allocation implies.  This variant keeps its split-K
- * scratch (the partial sums that the K chunks of a row pair exchange) in a fixed array that is
- * part of the library image: FQ_STATIC_SCRATCH_BYTES on every GPU that loads the library, held
- * until the process exits.  It calls no cudaMalloc / cudaFree and nothing that allocates.
+ * the device-wide synchronisation an allocation implies.  This variant keeps its scratch (the
+ * per-blob partial sums that two thread blocks exchange when they share a 32-row strip of the
+ * matrix) in a fixed array that is part of the library image: FQ_STATIC_SCRATCH_BYTES on every
+ * GPU that loads the library, held until the process exits.  It calls no cudaMalloc / cudaFree
+ * and nothing that allocates.
  *   - batch 1 only; x_dev fp16 [k_in], y_dev fp16 [n_out], 16-byte aligned, caller-owned.
- *   - Returns FQ_ERR_SCRATCH (and launches nothing) when the layer at its active width needs
- *     more scratch than the array holds: 256 bytes per (32-row pair x K chunk of 512..1536
- *     columns).  Every Llama-2-7B / 13B shaped layer fits.
+ *   - Returns FQ_ERR_SCRATCH (and launches nothing) when the layer needs more scratch than the
+ *     array holds: 256 bytes per (32-row strip x blob of 512 columns), i.e.
+ *     ceil(n_out / 32) * ceil(k_in / 512) * 256 bytes.  Every Llama-2-7B / 13B shaped layer fits.
  *   - The first call on a device looks up the array's device address (once per device, with
  *     that device current); make that first call before starting any stream capture.
  *   - All calls share the one array and it keeps whatever the last call left there.  Nothing
  *     in it has to be cleared: every partial sum carries the tag of the call that wrote it and
  *     is ignored under any other tag.  Two calls that overlap on the GPU (different streams,
- *     or different contexts) race on it: serialise them. */
+ *     or different contexts) race on it: serialise them.  Host calls are not thread-safe either:
+ *     the per-device tag counter and address cache are plain statics. */
 #define FQ_STATIC_SCRATCH_BYTES (2u << 20)
 int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);
 
@@ -199,8 +203,11 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
  *   phases_host (may be NULL = no ordering): non-decreasing int [n_ops], starting at 0 and
  *       without gaps; an op of phase p does not read its x before every op of phase p-1 has
  *       written its y (weights of later ops are prefetched meanwhile).
- * May grow the context's workspace (device allocation) when the op list is larger than
- * any seen before; otherwise enqueues one small host-to-device copy and one kernel. */
+ * Batch 1: at most 512 ops and 1024 phases per call (FQ_ERR_SHAPE otherwise).
+ * The call builds a table (ops, and which strips every thread block computes) and uploads it from a
+ * pinned buffer; a call with the same arguments under the same configuration reuses the uploaded
+ * table and only launches the kernel.  The workspace was sized by fq_pack_layer for lists that use
+ * every layer at most once; a list that repeats layers may grow it (device allocation + sync). */
 int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host,
                   const uint16_t* const* x_dev_host, uint16_t* const* y_dev_host,
                   const int* phases_host, int batch, void* stream);
@@ -234,6 +241,18 @@ int fq_active_bits(const fq_ctx* ctx, int layer);
 /* Synchronises the context's device, then returns and clears the device status word
  * (FQ_OK, or FQ_ERR_TIMEOUT if a bounded wait inside a kernel gave up). */
 int fq_status(fq_ctx* ctx);
+
+/* Limit of every device-side wait of the decode kernels, in nanoseconds (default 2e9; 0 restores the
+ * default).  Diagnostic support: with a limit shorter than any real wait a launch gives up at once,
+ * records FQ_ERR_TIMEOUT, drains its copies and returns; fq_status() then reports the code and resets
+ * the counters, and later launches are unaffected. */
+int fq_set_wait_limit_ns(fq_ctx* ctx, unsigned long long ns);
+
+/* Algorithmic sizes (the terms of the footprint, Sec. III): bytes of the b-bit codes of a layer,
+ * n_out * k_in * bits / 8, and of its scale/zero words, n_out * (k_in / group) * 4.  0 for invalid
+ * arguments.  (fq_store_bytes is the size of the stored variant including tile padding.) */
+size_t fq_code_bytes(int n_out, int k_in, int bits);
+size_t fq_meta_bytes(int n_out, int k_in, int group);
 const char* fq_strerror(int code);
 
 #ifdef __cplusplus

@@ -200,6 +200,25 @@ size_t fq_store_bytes(int n_out, int k_in, int bits, int fmt)
     return (size_t)store_bytes(n_out, k_in, bits);
 }
 
+size_t fq_code_bytes(int n_out, int k_in, int bits)
+{
+    if (n_out < 1 || k_in < 1 || k_in % kGroup != 0 || bits < 2 || bits > 8) return 0;
+    return (size_t)n_out * (size_t)k_in * (size_t)bits / 8u;
+}
+
+size_t fq_meta_bytes(int n_out, int k_in, int group)
+{
+    if (n_out < 1 || k_in < 1 || group != kGroup || k_in % kGroup != 0) return 0;
+    return (size_t)n_out * (size_t)(k_in / kGroup) * 4u;
+}
+
+int fq_set_wait_limit_ns(fq_ctx* ctx, unsigned long long ns)
+{
+    if (!ctx) return FQ_ERR_ARG;
+    ctx->wait_limit_ns = ns ? ns : 2000000000ull;
+    return FQ_OK;
+}
+
 int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int group,
                       uint8_t* codes_dev, uint16_t* scales_dev, uint16_t* zeros_dev, void* stream)
 {

@@ -28,6 +28,8 @@
 // loop, the producer waits for its copies in flight and the CTA returns.
 #include <cuda_fp16.h>
 
+#include <atomic>
+
 #include "fq_internal.cuh"
 #include "fq_ptx.cuh"
 #include "fq_gemv_core.cuh"
@@ -42,7 +44,7 @@ constexpr int kCW = 16;                                // consumer warps; consec
 constexpr int kKLanes = kCW;
 constexpr int kProducerWarp = kCW;
 constexpr int kPrepWarp = kCW + 1;                     // first activation pre-processing warp
-constexpr int kPrepWarps = 7;                          // 24 warps in all: 80 registers per thread
+constexpr int kPrepWarps = 8;                          // the eight blobs of a 4096-column activation vector convert side by side
 constexpr int kThreads = (kCW + 1 + kPrepWarps) * 32;
 constexpr int kStageBytes = 34816;                     // one unit: 4 x 4-bit blobs or 2 x 8-bit blobs
 constexpr int kBlobsMax = 6;                           // blobs per unit, at most (< kKLanes: a warp gets at most one item of a unit)
@@ -831,7 +833,7 @@ static int static_scratch_address(int device, unsigned char** out)
 // counter per device.
 int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t st)
 {
-    static unsigned epoch[64] = {};
+    static std::atomic<unsigned> epoch[64];      // one tag counter per device, shared by every context and host thread
     if (partial_bytes > FQ_STATIC_SCRATCH_BYTES) return FQ_ERR_SCRATCH;
     unsigned char* base = nullptr;
     const int rc = static_scratch_address(ctx->device, &base);
@@ -840,7 +842,9 @@ int launch_gemv_static(Ctx* ctx, GemvOp op, size_t partial_bytes, cudaStream_t s
     Args a{};
     a.status = ctx->status_dev;
     a.n_ops = 1;
-    a.epoch = next_epoch(epoch[ctx->device]);
+    unsigned e = epoch[ctx->device].fetch_add(1u) + 1u;
+    if (e == 0u) e = epoch[ctx->device].fetch_add(1u) + 1u;      // 0 marks words that no launch has written
+    a.epoch = e;
     a.wait_ns = ctx->wait_limit_ns;
     return launch(ctx, op, a, op.n_units, st);
 }

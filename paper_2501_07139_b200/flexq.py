@@ -23,6 +23,7 @@ EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
     "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load", "fq_search_chain", "fq_prune_chain", "fq_sqdiff",
+    "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes",
 ]
 
 
@@ -75,6 +76,11 @@ def lib():
     L.fq_storage_bytes.restype = u64
     L.fq_active_bits.argtypes = [vp, i]
     L.fq_status.argtypes = [vp]
+    L.fq_set_wait_limit_ns.argtypes = [vp, u64]
+    L.fq_code_bytes.argtypes = [i, i, i]
+    L.fq_code_bytes.restype = C.c_size_t
+    L.fq_meta_bytes.argtypes = [i, i, i]
+    L.fq_meta_bytes.restype = C.c_size_t
     L.fq_strerror.argtypes = [i]
     L.fq_strerror.restype = C.c_char_p
     for name in EXPORTS:
@@ -91,6 +97,14 @@ def fq_strerror(code: int) -> str:
 
 def fq_store_bytes(n_out: int, k_in: int, bits: int, fmt: int) -> int:
     return int(lib().fq_store_bytes(n_out, k_in, bits, fmt))
+
+
+def fq_code_bytes(n_out: int, k_in: int, bits: int) -> int:
+    return int(lib().fq_code_bytes(n_out, k_in, bits))
+
+
+def fq_meta_bytes(n_out: int, k_in: int, group: int = 128) -> int:
+    return int(lib().fq_meta_bytes(n_out, k_in, group))
 
 
 def _stream() -> int:
@@ -232,6 +246,10 @@ class FlexQ:
 
     def fq_status(self) -> int:
         return int(lib().fq_status(self._h))
+
+    def fq_set_wait_limit_ns(self, ns: int):
+        """Limit of every device-side wait of the decode kernels (0 restores the default of 2 s)."""
+        _check(lib().fq_set_wait_limit_ns(self._h, int(ns)), "fq_set_wait_limit_ns")
 
     # -- decode --------------------------------------------------------------------------
     def fq_gemv(self, layer: int, x: torch.Tensor, y: torch.Tensor):

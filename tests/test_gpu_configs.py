@@ -32,7 +32,7 @@ class _ParentRows:
     def __init__(self, cfg, shapes, rows_per_layer):
         self.rows, self.q8, self.s, self.z = [], [], [], []
         for i, sh in enumerate(shapes):
-            rows = S.sample_rows(5000 + i, sh.n_out, rows_per_layer)[:rows_per_layer + 2]
+            rows = S.sample_rows(5000 + i, sh.n_out, rows_per_layer)
             w = np.concatenate([S.weight_rows(S.tensor_key(cfg, i, S.TENSOR_W), int(r), int(r) + 1, sh.k_in).numpy()
                                 for r in rows])
             q8, s, z = O.quantize(w, 8)
@@ -57,7 +57,8 @@ def _check_decode(fq, shapes, ref, bits, xs, batch, tol):
         want = ref.gemv(i, int(bits[i]), bits_of(xs[i]))           # [batch][rows]
         got = got_all[:, ref.rows[i]]
         num += float(((got - want) ** 2).sum()); den += float((want ** 2).sum())
-        assert O.rel_l2(got, want) <= 3 * tol, (shapes[i].name, int(bits[i]))     # few rows per matrix
+        assert O.rel_l2(got, want) <= tol, (shapes[i].name, int(bits[i]))         # the stated tolerance, per matrix
+        assert np.max(np.abs(got - want)) <= 4 * tol * np.max(np.abs(want)), (shapes[i].name, int(bits[i]))
     assert np.sqrt(num / den) <= tol, np.sqrt(num / den)
 
 
@@ -70,7 +71,7 @@ def test_config2_7b_nested_chain():
     fq, stores = _build_nested(P, 2, shapes, device)
     assert fq.fq_storage_bytes() == O.footprint(n, k, [8] * L) == 6_678_380_544
     chain = S.config_chain(S.tensor_key(2, 0, S.TENSOR_CHAIN), shapes, 12, 7.0, 3.5, 3)
-    ref = _ParentRows(2, shapes, 2)
+    ref = _ParentRows(2, shapes, 58)
     xs = [S.activations(S.tensor_key(2, i, S.TENSOR_X), 1, sh.k_in).to(device) for i, sh in enumerate(shapes)]
     probe = [0, 100, 223]
     before = [stores[i].clone() for i in probe]
@@ -106,7 +107,7 @@ def test_config4_13b_nested_chain_decode_and_prefill():
     chain = S.config_chain(S.tensor_key(4, 0, S.TENSOR_CHAIN), shapes, 16, 6.0, 2.5, 2)
     for bits in chain:
         assert fq.fq_set_config([int(b) for b in bits]) == O.footprint(n, k, bits)
-    ref = _ParentRows(4, shapes, 1)
+    ref = _ParentRows(4, shapes, 26)
     x1 = [S.activations(S.tensor_key(4, i, S.TENSOR_X), 1, sh.k_in).to(device) for i, sh in enumerate(shapes)]
     x8 = [S.activations(S.tensor_key(4, 1000 + i, S.TENSOR_X), 8, sh.k_in).to(device) for i, sh in enumerate(shapes)]
     for ci in (0, 15):

@@ -31,7 +31,7 @@ def test_7b_stack_sampled_rows_match_oracle():
     for i, sh in enumerate(shapes):
         got_all = f64_of(ys[i])
         assert np.all(np.isfinite(got_all)), shapes[i].name
-        rows = S.sample_rows(1000 + i, sh.n_out, 6)
+        rows = S.sample_rows(1000 + i, sh.n_out, 58)            # 64 rows of every matrix
         # contiguous runs of rows are generated and quantised on the CPU, one row at a time
         w = np.concatenate([S.weight_rows(S.tensor_key(bench.CONFIG_ID, i, S.TENSOR_W), int(r), int(r) + 1,
                                           sh.k_in).numpy() for r in rows])
@@ -42,7 +42,8 @@ def test_7b_stack_sampled_rows_match_oracle():
         worst = max(worst, err)
         num += float(((got - ref) ** 2).sum())
         den += float((ref ** 2).sum())
-        assert err <= 2 * GEMV_TOL, (sh.name, int(bits[i]), err)      # few rows: looser per-sample bound
-    # pooled over all sampled rows of the stack the error must meet the stated tolerance
+        assert err <= GEMV_TOL, (sh.name, int(bits[i]), err)          # the stated tolerance, per matrix
+        # ... and no single output is off by more than a few times that (a norm alone would hide one bad row)
+        assert np.max(np.abs(got - ref)) <= 4 * GEMV_TOL * np.max(np.abs(ref)), (sh.name, int(bits[i]))
     assert np.sqrt(num / den) <= GEMV_TOL, (np.sqrt(num / den), worst)
     fq.fq_destroy()

@@ -118,6 +118,8 @@ def _gemv_case(P, fmt, bits, n, k, batch, cfg):
     assert np.all(np.isfinite(got))
     for b in range(batch):
         assert O.rel_l2(got[b], ref[b]) <= GEMV_TOL, (bits, b, O.rel_l2(got[b], ref[b]))
+        # element by element too: a norm alone would hide one bad row among a thousand
+        assert np.max(np.abs(got[b] - ref[b])) <= 4 * GEMV_TOL * np.max(np.abs(ref[b])), (bits, b)
     fq.fq_destroy()
     return codes, s, z
 
