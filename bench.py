@@ -52,8 +52,11 @@ def read_ncu_traffic(footprint_bytes):
     try:
         with open(os.path.join(ROOT, "profiles", "gemv_stack_traffic.json")) as f:
             d = json.load(f)
-        with open(os.path.join(ROOT, "paper_2501_07139_b200", "csrc", "fq_gemv.cu"), "rb") as f:
-            sha = hashlib.sha256(f.read()).hexdigest()
+        h = hashlib.sha256()
+        for name in ("fq_gemv1.cu", "fq_gemv_core.cuh"):                 # the batch-1 decode kernel and its arithmetic
+            with open(os.path.join(ROOT, "paper_2501_07139_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+        sha = h.hexdigest()
         if sha != d["source_sha256"]:
             return None, "kernel changed since the ncu capture"
         return d["ratio"] * footprint_bytes, d["note"]
@@ -192,11 +195,12 @@ def _time_ms(fn, steps, warmup=3):
     return e0.elapsed_time(e1) / steps
 
 
-def config_report(P, device, steps):
+def config_report(P, device, steps, brief=False):
     """The other workloads of the problem statement, one JSON object each (printed by --all-configs):
     config 0 (one 4096x4096 4-bit layer, rotated over copies larger than L2), config 2 (7B-shaped nested
     stack, 12-configuration chain) and config 4 (13B-shaped nested stack, 16 configurations, batch 1 / 8
-    decode and prefill at 2048 tokens)."""
+    decode and prefill at 2048 tokens).  brief: only the first, a middle and the last configuration of each
+    chain and no ensemble search -- what the default bench line carries in its `configs` object."""
     peaks, kind = measured_peaks()
     out = []
     # ---- config 0
@@ -244,8 +248,10 @@ def config_report(P, device, steps):
             args_dep = fq.stack_args(list(range(L)), xs, ys, phases)
             args_free = fq.stack_args(list(range(L)), xs, ys, None)
             for ci, bits in enumerate(chain):
+                if brief and ci not in ((0, n_cfg // 2 - 1, n_cfg - 1) if cfg == 2 else (0, n_cfg - 1)):
+                    continue
                 t0 = time.perf_counter()
-                if ci == 0 or batch != 1:
+                if ci == 0 or batch != 1 or brief:
                     fp = fq.fq_set_config([int(b) for b in bits])
                 else:                                            # the chain is one-way: every step is a transition
                     rep = fq.fq_transition([int(b) for b in bits], require_one_way=True)
@@ -259,15 +265,16 @@ def config_report(P, device, steps):
                 ms_free = _time_ms(lambda: fq.fq_gemv_stack_raw(args_free, batch), steps)
                 rows.append({"batch": batch, "config_index": ci, "average_bits": S.average_bits(bits, shapes),
                              "footprint_bytes": fp, "set_config_host_us": switch_us, "first_pass_ms": first_ms,
-                             "ms_per_pass": ms, "GBps": fp / ms / 1e6, "ms_unordered": ms_free, "GBps_unordered": fp / ms_free / 1e6})
+                             "ms_per_pass": ms, "GBps": fp / ms / 1e6, "frac": fp / ms / 1e6 / peaks["hbm_gbs"],
+                             "ms_unordered": ms_free, "GBps_unordered": fp / ms_free / 1e6})
             del xs, ys
         entry = {"config": cfg, "workload": f"{model}-shaped stack, nested bit-planes, {n_cfg}-configuration chain",
-                 "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0,
-                 "transitions": {"steps": len(steps_freed), "one_way": True, "bytes_loaded_total": int(sum(steps_loaded)),
-                                 "granularity_bytes_max": int(max(steps_freed)), "granularity_bytes_mean": float(np.mean(steps_freed)),
-                                 "note": "fq_transition per chain step: memory a deployment can release; nothing has to be loaded"},
-                 "decode": rows}
-        if cfg == 2:
+                 "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0, "decode": rows}
+        if steps_freed:
+            entry["transitions"] = {"steps": len(steps_freed), "one_way": True, "bytes_loaded_total": int(sum(steps_loaded)),
+                                    "granularity_bytes_max": int(max(steps_freed)), "granularity_bytes_mean": float(np.mean(steps_freed)),
+                                    "note": "fq_transition per chain step: memory a deployment can release; nothing has to be loaded"}
+        if cfg == 2 and not brief:
             # the offline side on the same stack: tables measured with the prefill kernel, tree search, pruning
             from paper_2501_07139_b200 import search as SR
             levels = [8, 5, 3]
@@ -346,6 +353,24 @@ def oracle_pass(items):
     return total_bytes, total_s
 
 
+def oracle_pass_threads(items, threads):
+    """The same pass with the rows of every matrix dealt to `threads` host threads (the oracle's C routine is
+    called once per row slice and releases the interpreter lock; the arithmetic of a row is unchanged)."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import fq_oracle as O
+    total_bytes, total_s = 0, 0.0
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        for codes, sc, zr, b, xb, nbytes in items:
+            n = codes.shape[0]
+            cuts = [n * t // threads for t in range(threads + 1)]
+            slices = [(codes[a:e], sc[a:e], zr[a:e]) for a, e in zip(cuts, cuts[1:]) if e > a]
+            t0 = time.perf_counter()
+            list(pool.map(lambda p: O.gemv(p[0], p[1], p[2], b, xb), slices))
+            total_s += time.perf_counter() - t0
+            total_bytes += nbytes
+    return total_bytes, total_s
+
+
 def oracle_desc(n_layers):
     return f"oracle GEMV over the first {n_layers} matrices of the stack ({n_layers / 7:.2g} blocks), single thread"
 
@@ -399,12 +424,13 @@ def main():
     ap.add_argument("--blocks", type=int, default=32, help="decoder blocks of the 7B-shaped stack (32 = full)")
     ap.add_argument("--ref-layers", type=int, default=7,
                     help="--impl reference: matrices per step at most (fewer when warmup + steps would pass the time budget)")
-    ap.add_argument("--cpu-layers", type=int, default=14, help="matrices the cpu_baseline leg times the CPU oracle on")
+    ap.add_argument("--cpu-layers", type=int, default=28, help="matrices the cpu_baseline leg times the CPU oracle on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill (tensor-core GEMM) leg")
     ap.add_argument("--prefill-steps", type=int, default=3)
     ap.add_argument("--prefill-tokens", type=int, default=PREFILL_TOKENS)
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill leg and print its object")
+    ap.add_argument("--no-configs", action="store_true", help="leave the `configs` object (configs 0, 2, 4 in brief) out of the line")
     ap.add_argument("--all-configs", action="store_true",
                     help="instead of the bench line, print one JSON object per other workload (configs 0, 2, 4)")
     args = ap.parse_args()
@@ -507,6 +533,19 @@ def main():
         return
 
     peaks, peak_kind = measured_peaks()
+    # a second denominator: what a read-only pass over 4 GiB reaches on this GPU right now
+    probe = torch.empty(1 << 30, dtype=torch.int32, device=device)
+    for _ in range(2):
+        fq.fq_stream_read(probe)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        fq.fq_stream_read(probe)
+    e1.record()
+    torch.cuda.synchronize()
+    stream_gbs = 5 * probe.numel() * 4 / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    del probe
     gbs = footprint / (ms * 1e-3) / 1e9
     traffic, traffic_note = read_ncu_traffic(footprint)
     line = {
@@ -531,7 +570,8 @@ def main():
             "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": gbs / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
             "frac_of_nominal_8TBs": gbs / 8000.0,
-            "kernel": "gemv_kernel<1> (one launch per pass; algorithmic bytes = footprint of the configuration)",
+            "kernel": "gemv1_kernel (one launch per pass; algorithmic bytes = footprint of the configuration)",
+            "stream_read_gbs": stream_gbs, "frac_of_stream_read": gbs / stream_gbs,
             "traffic": traffic, "traffic_note": traffic_note,
         },
         "clocks": clocks,
@@ -552,11 +592,18 @@ def main():
                          "frac_of_burst": pf["tflops"] / burst, "traffic": None,
                          "kernel": "gemm_kernel (tcgen05) + dequant_kernel; flops = 2*M*N*K per matrix"},
         }
+    if not args.no_configs and world == 1 and args.blocks == 32:
+        line["configs"] = config_report(P, device, 5, brief=True)
     if not args.no_cpu_baseline:
         n_layers = min(args.cpu_layers, L)
-        byts, secs = oracle_pass(oracle_inputs(shapes, bits, n_layers, device))
-        line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": oracle_desc(n_layers)}
+        items = oracle_inputs(shapes, bits, n_layers, device)
+        cores = len(os.sched_getaffinity(0))
+        byts1, secs1 = oracle_pass(items[:min(7, n_layers)])
+        byts, secs = oracle_pass_threads(items, cores)
+        line["cpu_baseline"] = {"value": byts / secs / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": oracle_desc(n_layers).replace("single thread", f"rows of each matrix dealt to {cores} host threads"),
+                                "single_thread": {"value": byts1 / secs1 / 1e9, "unit": UNIT, "cores": 1,
+                                                  "sample": oracle_desc(min(7, n_layers))}}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

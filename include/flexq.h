@@ -248,6 +248,11 @@ int fq_status(fq_ctx* ctx);
  * the counters, and later launches are unaffected. */
 int fq_set_wait_limit_ns(fq_ctx* ctx, unsigned long long ns);
 
+/* Measurement support: one read-only pass over `bytes` of device memory (16-byte aligned) with vector loads,
+ * enqueued on `stream`.  Timing it gives the streaming-read bandwidth of the part, the ceiling of a kernel
+ * that, like the decode path, reads weights once and writes almost nothing. */
+int fq_stream_read(fq_ctx* ctx, const void* src_dev, size_t bytes, void* stream);
+
 /* Algorithmic sizes (the terms of the footprint, Sec. III): bytes of the b-bit codes of a layer,
  * n_out * k_in * bits / 8, and of its scale/zero words, n_out * (k_in / group) * 4.  0 for invalid
  * arguments.  (fq_store_bytes is the size of the stored variant including tile padding.) */

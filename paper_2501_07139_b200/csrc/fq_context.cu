@@ -212,6 +212,15 @@ size_t fq_meta_bytes(int n_out, int k_in, int group)
     return (size_t)n_out * (size_t)(k_in / kGroup) * 4u;
 }
 
+int fq_stream_read(fq_ctx* ctx, const void* src_dev, size_t bytes, void* stream)
+{
+    if (!ctx || !src_dev || bytes < 16) return FQ_ERR_ARG;
+    if (!aligned(src_dev, 16)) return FQ_ERR_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    return launch_stream_read(src_dev, bytes, reinterpret_cast<unsigned*>(ctx->ws + 8 * 4096 + 32), ctx->sm_count, (cudaStream_t)stream);
+}
+
 int fq_set_wait_limit_ns(fq_ctx* ctx, unsigned long long ns)
 {
     if (!ctx) return FQ_ERR_ARG;

@@ -149,9 +149,45 @@ struct FieldLoop {
     }
 };
 
+// The same with the (superstep, tile) index known only at run time: one multiply-add per field instead of an
+// immediate offset, but the loop over supersteps and tiles need not be unrolled.
+template <int VARIANT, int FI, int PREFIX>
+struct FieldLoopRt {
+    static __device__ __forceinline__ void run(uint32_t fbase, int st, const uint4 (&bx)[4], int c, int m1, int (&v)[2][2])
+    {
+        constexpr FieldList FL = variant_fields(VARIANT);
+        if constexpr (FI < FL.n) {
+            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
+            field_step<F, SHIFT, FI == 0, kBlobSteps * kBlobTiles * 512 * PREFIX>(fbase + st * (F * 512), bx, c, m1, v);
+            FieldLoopRt<VARIANT, FI + 1, PREFIX + F>::run(fbase, st, bx, c, m1, v);
+        }
+    }
+};
+
+// Group epilogue of one (superstep, tile): y += s * 2^-e * (v - (z - adjust) * sum x_int).
+template <int ADJUST>
+__device__ __forceinline__ void group_epilogue(const uint4 mw, const int (&v)[2][2], const int (&nx)[2], const float (&sc)[2],
+                                               float (&tot)[2])
+{
+    const uint32_t mm[2][2] = {{mw.x, mw.y}, {mw.z, mw.w}};      // (grp 0: row g, g + 8), (grp 1: row g, g + 8)
+#pragma unroll
+    for (int grp = 0; grp < 2; grp++) {
+        const int base = ADJUST ? -ADJUST * nx[grp] : 0;
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+            const uint32_t m = mm[grp][r];
+            const float s = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
+            const int t = v[grp][r] + (int)__umulhi(m, 65536u) * nx[grp] + base;
+            tot[r] = fmaf((float)t, s * sc[grp], tot[r]);
+        }
+    }
+}
+
 // One blob (32 rows x 512 columns): tot[tile][r] += dequantised dot products of rows 16 tile + g + 8 r (this
 // lane's step class only; the four lanes of a quad add up to the row sums).  Both row tiles share the B
-// registers and the group sums of the activations.
+// registers and the group sums of the activations.  Variants with one or two fields are unrolled over the
+// two supersteps and the two tiles; the others (up to seven fields) loop, or the fourteen specialised
+// bodies would not fit the instruction cache.
 //   blob : shared address of the blob          xd : this lane's B source per step class (digits or zeros)
 //   xg   : shared address of the blob's group sums / scales
 template <int VARIANT>
@@ -160,38 +196,51 @@ __device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)
     // a nested child reads the parent's top bits; the dropped bits are filled with their mid-point, which
     // is the same as lowering every zero point by that amount
     constexpr int kAdjust = (VARIANT >= 7 && VARIANT < 13) ? 1 << (7 - (VARIANT - 5)) : 0;
+    constexpr bool kUnrolled = variant_fields(VARIANT).n <= 2;
     const int g = lane >> 2, c = lane & 3;
     const uint32_t fbase = blob + kBlobMetaBytes + lane * 16;
     const uint32_t mbase = blob + g * 16;
     const int m1 = opaque_minus_one();
     const int czero = c == 0 ? m1 : 0;                         // only the class-0 lane of a quad subtracts the zero-point term
-    static_for<0, kBlobSteps>([&](auto SSI) {
-        constexpr int ss = decltype(SSI)::value;
-        uint4 bx[4];
-        static_for<0, 4>([&](auto JC) { bx[decltype(JC)::value] = lds128<ss * 512>(xd[decltype(JC)::value]); });
-        const uint2 xs2 = lds64<ss * 8>(xg), sc2 = lds64<16 + ss * 8>(xg);
-        const int nx[2] = {(int)xs2.x * czero, (int)xs2.y * czero};
-        const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
-        static_for<0, kBlobTiles>([&](auto TLI) {
-            constexpr int tile = decltype(TLI)::value;
-            const uint4 mw = lds128<(ss * kBlobTiles + tile) * 128>(mbase);   // (grp 0: row g, g + 8), (grp 1: row g, g + 8)
-            int v[2][2];
-            FieldLoop<VARIANT, 0, 0, ss, tile>::run(fbase, bx, c, m1, v);
-            // group epilogue: y += s * 2^-e * (v - (z - adjust) * sum x_int)
-            const uint32_t mm[2][2] = {{mw.x, mw.y}, {mw.z, mw.w}};
-#pragma unroll
-            for (int grp = 0; grp < 2; grp++) {
-                const int base = kAdjust ? -kAdjust * nx[grp] : 0;
-#pragma unroll
-                for (int r = 0; r < 2; r++) {
-                    const uint32_t m = mm[grp][r];
-                    const float s = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
-                    const int t = v[grp][r] + (int)__umulhi(m, 65536u) * nx[grp] + base;
-                    tot[tile][r] = fmaf((float)t, s * sc[grp], tot[tile][r]);
-                }
-            }
+    if constexpr (kUnrolled) {
+        static_for<0, kBlobSteps>([&](auto SSI) {
+            constexpr int ss = decltype(SSI)::value;
+            uint4 bx[4];
+            static_for<0, 4>([&](auto JC) { bx[decltype(JC)::value] = lds128<ss * 512>(xd[decltype(JC)::value]); });
+            const uint2 xs2 = lds64<ss * 8>(xg), sc2 = lds64<16 + ss * 8>(xg);
+            const int nx[2] = {(int)xs2.x * czero, (int)xs2.y * czero};
+            const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
+            static_for<0, kBlobTiles>([&](auto TLI) {
+                constexpr int tile = decltype(TLI)::value;
+                const uint4 mw = lds128<(ss * kBlobTiles + tile) * 128>(mbase);
+                int v[2][2];
+                FieldLoop<VARIANT, 0, 0, ss, tile>::run(fbase, bx, c, m1, v);
+                group_epilogue<kAdjust>(mw, v, nx, sc, tot[tile]);
+            });
         });
-    });
+    } else {
+#pragma unroll 1
+        for (int ss = 0; ss < kBlobSteps; ss++) {
+            uint4 bx[4];
+            static_for<0, 4>([&](auto JC) { bx[decltype(JC)::value] = lds128(xd[decltype(JC)::value] + ss * 512); });
+            const uint2 xs2 = lds64(xg + ss * 8), sc2 = lds64<16>(xg + ss * 8);
+            const int nx[2] = {(int)xs2.x * czero, (int)xs2.y * czero};
+            const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
+            float tt[kBlobTiles][2] = {{tot[0][0], tot[0][1]}, {tot[1][0], tot[1][1]}};
+#pragma unroll 1
+            for (int tile = 0; tile < kBlobTiles; tile++) {
+                const int st = ss * kBlobTiles + tile;
+                const uint4 mw = lds128(mbase + st * 128);
+                int v[2][2];
+                FieldLoopRt<VARIANT, 0, 0>::run(fbase, st, bx, c, m1, v);
+                float t2[2] = {0.f, 0.f};
+                group_epilogue<kAdjust>(mw, v, nx, sc, t2);
+                if (tile == 0) { tt[0][0] += t2[0]; tt[0][1] += t2[1]; }
+                else { tt[1][0] += t2[0]; tt[1][1] += t2[1]; }
+            }
+            tot[0][0] = tt[0][0]; tot[0][1] = tt[0][1]; tot[1][0] = tt[1][0]; tot[1][1] = tt[1][1];
+        }
+    }
 }
 
 // Selects the specialised loop of a variant (variant_index in fq_layout.cuh).

@@ -103,6 +103,8 @@ int launch_export_planes(const void* store, int n_out, int k_in, int bits, const
 int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, uint16_t* scales, uint16_t* zeros,
                        cudaStream_t st);
 
+int launch_stream_read(const void* src, size_t bytes, unsigned* sink, int sm_count, cudaStream_t st);
+
 // Chunking policy of the decode kernel: k blobs (512 columns) per K chunk.
 int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_bytes_per_unit(int batch);

@@ -298,4 +298,30 @@ int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, 
     return FQ_OK;
 }
 
+// ------------------------------------------------------------------------------- streaming read (measurement)
+// Reads a buffer once with 16-byte loads, four in flight per thread, and folds the words into one value per
+// thread block: what a kernel that only READS memory (as the decode path does) can reach on this part.
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4* __restrict__ src, long long n16, unsigned* sink)
+{
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned acc = 0u;
+    for (; i + 3 * stride < n16; i += 4 * stride) {
+        const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride), d = __ldcs(src + i + 3 * stride);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+    }
+    for (; i < n16; i += stride) {
+        const uint4 a = __ldcs(src + i);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w;
+    }
+    for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0 && acc == 0x9e3779b9u) atomicXor(sink, acc);      // (keeps the loads alive; practically never taken)
+}
+
+int launch_stream_read(const void* src, size_t bytes, unsigned* sink, int sm_count, cudaStream_t st)
+{
+    stream_read_kernel<<<sm_count * 4, 512, 0, st>>>(static_cast<const uint4*>(src), (long long)(bytes / 16), sink);
+    return cudaGetLastError() == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;
+}
+
 }  // namespace fq

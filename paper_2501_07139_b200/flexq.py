@@ -23,7 +23,7 @@ EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
     "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load", "fq_search_chain", "fq_prune_chain", "fq_sqdiff",
-    "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes",
+    "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes", "fq_stream_read",
 ]
 
 
@@ -77,6 +77,7 @@ def lib():
     L.fq_active_bits.argtypes = [vp, i]
     L.fq_status.argtypes = [vp]
     L.fq_set_wait_limit_ns.argtypes = [vp, u64]
+    L.fq_stream_read.argtypes = [vp, vp, C.c_size_t, vp]
     L.fq_code_bytes.argtypes = [i, i, i]
     L.fq_code_bytes.restype = C.c_size_t
     L.fq_meta_bytes.argtypes = [i, i, i]
@@ -246,6 +247,10 @@ class FlexQ:
 
     def fq_status(self) -> int:
         return int(lib().fq_status(self._h))
+
+    def fq_stream_read(self, buf: torch.Tensor):
+        """One read-only pass over a device buffer (measurement support)."""
+        _check(lib().fq_stream_read(self._h, buf.data_ptr(), buf.numel() * buf.element_size(), _stream()), "fq_stream_read")
 
     def fq_set_wait_limit_ns(self, ns: int):
         """Limit of every device-side wait of the decode kernels (0 restores the default of 2 s)."""

@@ -85,6 +85,19 @@ def test_quantizer_hand_worked_group():
     assert z[0, 0] == 0x4600                       # fp16(6.0)
 
 
+def test_quantizer_rounds_the_scale_before_the_codes():
+    # b = 4, mn = 0, mx = 1: (mx - mn) / 15 = 0.0666... is not an fp16 number.  Between 2^-4 and 2^-3 fp16
+    # steps by 2^-14; 0.0666667 = 2^-4 + 68.27 * 2^-14 rounds to 2^-4 + 68 * 2^-14 = 0.066650390625 = 0x2C44.
+    # The codes are computed against THAT scale: 0.4999 / 0.066650390625 = 7.5003 -> 8, whereas against the
+    # unrounded 1/15 it would be 7.4985 -> 7.  (z = rint(0 / s) = 0.)
+    w = np.full((1, 128), 0.25, np.float32)        # 0.25 / s = 3.7509 -> 4 either way
+    w[0, 0], w[0, 1], w[0, 2] = 0.0, 1.0, 0.4999
+    codes, s, z = O.quantize(w, 4)
+    assert s[0, 0] == 0x2C44 and z[0, 0] == 0x0000
+    assert codes[0, 0] == 0 and codes[0, 1] == 15 and codes[0, 2] == 8
+    assert np.all(codes[0, 3:] == 4)
+
+
 def test_quantizer_degenerate_and_clamped_groups():
     w = np.full((2, 128), 0.25, np.float32)        # constant group: range 0 -> s = 2^-14
     w[1] = 0.0
