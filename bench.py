@@ -163,23 +163,32 @@ def prefill_pass(P, device, blocks, steps, warmup, tokens=PREFILL_TOKENS):
         for i, sh in enumerate(shapes):
             fq.fq_gemm(i, xs[sh.k_in], ys[sh.n_out])
 
-    for _ in range(warmup):
-        one_pass()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one_pass()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
+    def one_pass_two():                             # the comparison point: dequantise to bf16, then a plain tcgen05 GEMM
+        for i, sh in enumerate(shapes):
+            fq.fq_gemm_two_pass(i, xs[sh.k_in], ys[sh.n_out])
+
+    def timed(fn):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    ms = timed(one_pass)
+    ms_two = timed(one_pass_two)
     status = fq.fq_status()
     fq.fq_destroy()
     if status != 0:
         raise RuntimeError(f"device status {status} after the prefill pass")
     flop = sum(2.0 * m * sh.n_out * sh.k_in for sh in shapes)
     return {"ms_per_pass": ms, "tflops": flop / (ms * 1e-3) / 1e12, "flop_per_pass": flop, "tokens": m,
-            "matrices": L, "average_bits": S.average_bits(bits, shapes), "gpu_launches_per_pass": 2 * L}
+            "matrices": L, "average_bits": S.average_bits(bits, shapes), "gpu_launches_per_pass": L,
+            "two_pass": {"ms_per_pass": ms_two, "tflops": flop / (ms_two * 1e-3) / 1e12, "gpu_launches_per_pass": 2 * L}}
 
 
 def _time_ms(fn, steps, warmup=3):
@@ -585,12 +594,14 @@ def main():
         line["prefill"] = {
             "metric": "prefill dequant-GEMM TFLOP/s", "value": pf["tflops"], "unit": "TFLOP/s", "ms_per_pass": pf["ms_per_pass"],
             "workload": f"bf16 activations {pf['tokens']} tokens through {pf['matrices']} matrices of the 7B-shaped stack, "
-                        f"bits seeded from {PREFILL_BITS} (average {pf['average_bits']:.2f}), one fq_gemm per matrix",
+                        f"bits seeded from {PREFILL_BITS} (average {pf['average_bits']:.2f}), one fq_gemm (fused kernel) per matrix",
             "dtype": "bf16", "gpu_launches_per_pass": pf["gpu_launches_per_pass"],
             "roofline": {"bound": "tensor", "achieved": pf["tflops"], "peak": sustained, "unit": "TFLOP/s",
                          "frac": pf["tflops"] / sustained, "peak_kind": f"of {peak_kind} (sustained bf16, the pass is a long step)",
                          "frac_of_burst": pf["tflops"] / burst, "traffic": None,
-                         "kernel": "gemm_kernel (tcgen05) + dequant_kernel; flops = 2*M*N*K per matrix"},
+                         "kernel": "gemm_fused_kernel (tcgen05; blobs dequantised inside); flops = 2*M*N*K per matrix"},
+            "two_pass": dict(pf["two_pass"], note="comparison point: dequant_kernel + gemm_kernel (fq_gemm_two_pass)",
+                             frac=pf["two_pass"]["tflops"] / sustained),
         }
     if not args.no_configs and world == 1 and args.blocks == 32:
         line["configs"] = config_report(P, device, 5, brief=True)

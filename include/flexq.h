@@ -215,12 +215,20 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host,
 /* Prefill / calibration-set evaluation (Sec. III-B: every candidate EQM is run forward over
  * token sequences):  Y[m][n] = sum_k X[m][k] * w^[n][k].
  *   X_dev bf16 [M][ldx >= k_in], Y_dev bf16 [M][ldy >= n_out], row-major, 16-byte aligned,
- *   ldx and ldy multiples of 8, 1 <= M <= 2^20.  The layer is dequantised to bf16 (one rounding of
- *   the exact (q - z) * s) into a workspace of n_out*k_in*2 bytes that the context owns (grown with
- *   a device allocation when a larger layer is first used), then multiplied on the tensor cores
- *   (tcgen05, fp32 accumulation in TMEM).  Enqueues two kernels on `stream`. */
+ *   ldx and ldy multiples of 8, 1 <= M <= 2^20.
+ * One fused kernel: X tiles arrive by TMA, the stored blobs are dequantised inside the kernel
+ * (w^ = (q - z) * s exactly in fp32, rounded once to bf16) into the shared-memory operand tiles of
+ * the tensor cores (tcgen05, fp32 accumulation in TMEM), Y is rounded once to bf16.  No workspace,
+ * no allocation; enqueues one kernel on `stream` and encodes one tensor map on the host. */
 int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx,
             uint16_t* Y_dev, int ldy, void* stream);
+
+/* The same product computed in two passes, kept as the comparison point of the fused kernel: the
+ * layer is first dequantised to bf16 into a workspace of n_out*k_in*2 bytes that the context owns
+ * (grown with a device allocation when a larger layer is first used), then multiplied by a plain
+ * tcgen05 GEMM.  Same arguments, same rounding points, same results up to the fp32 summation order. */
+int fq_gemm_two_pass(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx,
+                     uint16_t* Y_dev, int ldy, void* stream);
 
 /* Test / reporting support ------------------------------------------------------------ */
 

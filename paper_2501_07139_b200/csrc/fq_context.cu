@@ -662,7 +662,8 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
                       : launch_gemv_stack(ctx, ctx->stack_hdr, ctx->stack_dev, batch, st);
 }
 
-int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)
+static int gemm_common(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream,
+                       bool fused)
 {
     if (!ctx || !X_dev || !Y_dev) return FQ_ERR_ARG;
     if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
@@ -675,6 +676,11 @@ int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint1
     if (!v) return FQ_ERR_NO_VARIANT;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
+    const int zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
+    const int stride = blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits);
+    if (fused)
+        return launch_gemm_fused(ctx, v->store, stride, active_fields(L, bits), zero_adjust, L.n_out, L.k_in, X_dev, M, ldx,
+                                 Y_dev, ldy, (cudaStream_t)stream);
     const size_t need = (size_t)L.n_out * L.k_in * 2;
     if (need > ctx->gemm_ws_bytes) {
         FQ_CUDA_OK(cudaDeviceSynchronize());
@@ -683,9 +689,18 @@ int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint1
         FQ_CUDA_OK(cudaMalloc(&ctx->gemm_ws, need));
         ctx->gemm_ws_bytes = need;
     }
-    const int zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
-    return launch_gemm(ctx, v->store, blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits), active_fields(L, bits), zero_adjust,
-                       L.n_out, L.k_in, X_dev, M, ldx, Y_dev, ldy, ctx->gemm_ws, (cudaStream_t)stream);
+    return launch_gemm(ctx, v->store, stride, active_fields(L, bits), zero_adjust, L.n_out, L.k_in, X_dev, M, ldx, Y_dev, ldy,
+                       ctx->gemm_ws, (cudaStream_t)stream);
+}
+
+int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)
+{
+    return gemm_common(ctx, layer, X_dev, M, ldx, Y_dev, ldy, stream, true);
+}
+
+int fq_gemm_two_pass(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx, uint16_t* Y_dev, int ldy, void* stream)
+{
+    return gemm_common(ctx, layer, X_dev, M, ldx, Y_dev, ldy, stream, false);
 }
 
 int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* stream)

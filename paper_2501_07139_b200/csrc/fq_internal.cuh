@@ -109,6 +109,8 @@ int launch_stream_read(const void* src, size_t bytes, unsigned* sink, int sm_cou
 int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_bytes_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                 // batch 2..8
+int launch_gemm_fused(Ctx* ctx, const void* store, int blob_stride, const FieldList& fl, int zero_adjust, int n_out, int k_in,
+                      const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, cudaStream_t st);
 struct CtaWork;
 int launch_gemv1_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                // batch 1
 // table_dev: [GemvOp x n_ops][int phase_total x max(n_phases,1)][uint2 strips x sm_count x n_ops]

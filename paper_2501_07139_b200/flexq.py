@@ -23,7 +23,7 @@ EXPORTS = [
     "fq_create", "fq_destroy", "fq_store_bytes", "fq_quantize_layer", "fq_pack_layer",
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
     "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load", "fq_search_chain", "fq_prune_chain", "fq_sqdiff",
-    "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes", "fq_stream_read",
+    "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes", "fq_stream_read", "fq_gemm_two_pass",
 ]
 
 
@@ -70,6 +70,7 @@ def lib():
     L.fq_gemv_static.argtypes = [vp, i, vp, vp, vp]
     L.fq_gemv_stack.argtypes = [vp, i, vp, vp, vp, vp, i, vp]
     L.fq_gemm.argtypes = [vp, i, vp, i, i, vp, i, vp]
+    L.fq_gemm_two_pass.argtypes = [vp, i, vp, i, i, vp, i, vp]
     L.fq_export_layer.argtypes = [vp, i, i, vp, vp]
     L.fq_export_meta.argtypes = [vp, i, i, vp, vp, vp]
     L.fq_storage_bytes.argtypes = [vp]
@@ -300,6 +301,13 @@ class FlexQ:
         assert X.dtype == torch.bfloat16 and Y.dtype == torch.bfloat16
         _check(lib().fq_gemm(self._h, layer, X.data_ptr(), X.shape[0], X.stride(0), Y.data_ptr(), Y.stride(0),
                              _stream()), "fq_gemm")
+        return Y
+
+    def fq_gemm_two_pass(self, layer: int, X: torch.Tensor, Y: torch.Tensor):
+        """The comparison point of fq_gemm: dequantise to a bf16 workspace, then a plain tcgen05 GEMM."""
+        assert X.dtype == torch.bfloat16 and Y.dtype == torch.bfloat16
+        _check(lib().fq_gemm_two_pass(self._h, layer, X.data_ptr(), X.shape[0], X.stride(0), Y.data_ptr(), Y.stride(0),
+                                      _stream()), "fq_gemm_two_pass")
         return Y
 
     # -- export (tests / reporting) ----------------------------------------------------------

@@ -1,4 +1,5 @@
-"""GPU parity of the prefill path (fq_gemm, tcgen05 tensor-core GEMM) against the fp64 CPU oracle."""
+"""GPU parity of the prefill path against the fp64 CPU oracle: the fused kernel behind fq_gemm (blobs
+dequantised inside the tcgen05 GEMM) and its two-pass comparison point fq_gemm_two_pass."""
 import numpy as np
 import pytest
 import torch
@@ -17,6 +18,15 @@ def P():
     return P
 
 
+@pytest.fixture(params=["fused", "two_pass"])
+def which(request):
+    return request.param
+
+
+def _gemm(fq, which, layer, x, y):
+    return fq.fq_gemm(layer, x, y) if which == "fused" else fq.fq_gemm_two_pass(layer, x, y)
+
+
 def _ref(codes, s, z, bits, fmt, x):
     if fmt == 1:
         return O.gemm(codes >> (8 - bits), s, z, bits, bits_of(x), parent_bits=8)
@@ -24,7 +34,7 @@ def _ref(codes, s, z, bits, fmt, x):
 
 
 @pytest.mark.parametrize("fmt_bits", [(0, 2), (0, 3), (0, 4), (0, 5), (0, 6), (0, 7), (0, 8), (1, 3), (1, 6), (1, 8)])
-def test_gemm_small_every_element(P, fmt_bits):
+def test_gemm_small_every_element(P, which, fmt_bits):
     fmt, bits = fmt_bits
     n, k, m = 300, 384, 200                      # ragged against the 128 x 256 x 64 tiles
     stored = 8 if fmt == 1 else bits
@@ -34,7 +44,7 @@ def test_gemm_small_every_element(P, fmt_bits):
     fq.fq_set_config([bits])
     x = x_bf16(110, bits, m, k).cuda()
     y = torch.full((m, n + 4), float("nan"), dtype=torch.bfloat16, device="cuda")[:, :]   # ldy = n + 4 (multiple of 8)
-    fq.fq_gemm(0, x, y)
+    _gemm(fq, which, 0, x, y)
     assert fq.fq_status() == 0
     got = f64_of(y)[:, :n]
     ref = _ref(codes, s, z, bits, fmt, x)
@@ -48,14 +58,14 @@ def test_gemm_small_every_element(P, fmt_bits):
 
 
 @pytest.mark.parametrize("m", [1, 127, 129, 600])
-def test_gemm_token_counts(P, m):
+def test_gemm_token_counts(P, which, m):
     n, k = 512, 1024
     codes, s, z = make_layer(111, 0, n, k, 4)
     fq = P.FlexQ(1)
     fq.fq_pack_layer(0, *to_dev(codes, s, z), 4, P.FQ_FMT_PACKED)
     x = x_bf16(111, m, m, k).cuda()
     y = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
-    fq.fq_gemm(0, x, y)
+    _gemm(fq, which, 0, x, y)
     assert fq.fq_status() == 0
     rows = sorted(set([0, m - 1, m // 2, min(m - 1, 127), min(m - 1, 128)]))
     ref = O.gemm(codes, s, z, 4, bits_of(x[rows]))
@@ -63,7 +73,7 @@ def test_gemm_token_counts(P, m):
     fq.fq_destroy()
 
 
-def test_gemm_identity_probe_recovers_weights(P):
+def test_gemm_identity_probe_recovers_weights(P, which):
     """X = identity rows: Y[m][n] = bf16(w^[n][m]); checks operand orientation and every k position."""
     n, k = 256, 256
     codes, s, z = make_layer(112, 0, n, k, 8)
@@ -71,7 +81,7 @@ def test_gemm_identity_probe_recovers_weights(P):
     fq.fq_pack_layer(0, *to_dev(codes, s, z), 8, P.FQ_FMT_PACKED)
     x = torch.eye(k, dtype=torch.bfloat16, device="cuda")
     y = torch.empty((k, n), dtype=torch.bfloat16, device="cuda")
-    fq.fq_gemm(0, x, y)
+    _gemm(fq, which, 0, x, y)
     S_ = np.repeat(s.view(np.float16).astype(np.float64), 128, axis=1)
     Z_ = np.repeat(z.view(np.float16).astype(np.float64), 128, axis=1)
     exact = (codes.astype(np.float64) - Z_) * S_                       # [n][k], exact products
@@ -80,7 +90,7 @@ def test_gemm_identity_probe_recovers_weights(P):
     fq.fq_destroy()
 
 
-def test_gemm_7b_block_at_prefill_size_sampled(P):
+def test_gemm_7b_block_at_prefill_size_sampled(P, which):
     """First block of the 7B-shaped stack at M = 4 x 2048 tokens, bits from {2,3,4,6,8}: sampled outputs."""
     shapes = S.stack_shapes("7b", 1)
     bits = S.draw_bits(S.tensor_key(3, 0, S.TENSOR_BITS), len(shapes), [2, 3, 4, 6, 8])
@@ -98,7 +108,7 @@ def test_gemm_7b_block_at_prefill_size_sampled(P):
     for i, sh in enumerate(shapes):
         x = xs[sh.k_in]
         y = torch.empty((m, sh.n_out), dtype=torch.bfloat16, device="cuda")
-        fq.fq_gemm(i, x, y)
+        _gemm(fq, which, i, x, y)
         assert fq.fq_status() == 0
         trows = sorted(set([0, 127, 128, m - 1] + rng.integers(0, m, 12).tolist()))
         nrows = S.sample_rows(2000 + i, sh.n_out, 40)
