@@ -126,8 +126,8 @@ static __device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t
 }
 
 // Four codes of one row (one A register) -> four bf16 weights w^ = (q - z) * s, each rounded once.
-//   A byte q under the exponent byte 0x64 is the fp16 number 1024 + q; subtracting zz = 1024 + z in fp16 is
-//   exact (integers below 2048), the product with the fp16 scale is exact in fp32 (9 x 11 bits).
+//   Codes up to 255: a byte q under the exponent byte 0x64 is the fp16 number 1024 + q; subtracting zz = 1024 + z
+//   in fp16 is exact (integers below 2048), the product with the fp16 scale is exact in fp32 (9 x 11 bits).
 static __device__ __forceinline__ uint2 codes_to_bf16(uint32_t q4, __half2 zz, float s)
 {
     const uint32_t p02 = (q4 & 0x00ff00ffu) | 0x64006400u;          // columns 0 and 2
@@ -141,6 +141,21 @@ static __device__ __forceinline__ uint2 codes_to_bf16(uint32_t q4, __half2 zz, f
     o.y = *reinterpret_cast<const uint32_t*>(&hi);
     return o;
 }
+//   Codes below 128: a byte q in bits 16..22 under the exponent byte 0x43 is the fp32 number 128 + q, and
+//   fma(128 + q, s, c) with c = -(128 + z) * s (exact: 8 x 11 bits) is (q - z) * s without any rounding.
+static __device__ __forceinline__ uint2 small_codes_to_bf16(uint32_t q4, float c, float s)
+{
+    const float f0 = __uint_as_float(__byte_perm(q4, 0x43000000u, 0x7044));
+    const float f1 = __uint_as_float(__byte_perm(q4, 0x43000000u, 0x7144));
+    const float f2 = __uint_as_float(__byte_perm(q4, 0x43000000u, 0x7244));
+    const float f3 = __uint_as_float(__byte_perm(q4, 0x43000000u, 0x7344));
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(fmaf(f0, s, c), fmaf(f1, s, c));
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(fmaf(f2, s, c), fmaf(f3, s, c));
+    uint2 o;
+    o.x = *reinterpret_cast<const uint32_t*>(&lo);
+    o.y = *reinterpret_cast<const uint32_t*>(&hi);
+    return o;
+}
 
 template <int VARIANT>
 __global__ void __launch_bounds__(kFThreads, 1)
@@ -148,6 +163,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
 {
     constexpr FieldList FL = variant_fields(VARIANT);
     constexpr int kLoads = fields_loads(FL, FL.n);
+    constexpr bool kSmallCodes = VARIANT < 6;            // PACKED 2..7 bits: codes below 128, no zero adjustment
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -254,7 +270,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, local++) {
             const int mb = t % m_blocks, nb = t / m_blocks;
-            if (!g_wait(tfull, (uint32_t)local & 1u, abort_flag)) { ok = false; break; }
+            if (!g_wait<256>(tfull, (uint32_t)local & 1u, abort_flag)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
             for (int h = 0; h < 2; h++) {
@@ -347,18 +363,19 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                     merge_codes<VARIANT>(raw[tl], j0, code);
                     const uint32_t mm[2] = {meta[tl].x, meta[tl].y};
                     __half2 zz[2];
-                    float sc[2];
+                    float sc[2], cc[2];
 #pragma unroll
                     for (int hr = 0; hr < 2; hr++) {
                         sc[hr] = have ? __half2float(__ushort_as_half((unsigned short)(mm[hr] & 0xffffu))) : 0.f;   // rows past N: zeros
                         zz[hr] = __half2half2(__int2half_rn(1024 + (int)(mm[hr] >> 16) - a.zero_adjust));
+                        cc[hr] = -(float)(128 + (int)(mm[hr] >> 16)) * sc[hr];
                     }
 #pragma unroll
                     for (int jj = 0; jj < 2; jj++)
 #pragma unroll
                         for (int r = 0; r < 4; r++) {
                             const int hr = r & 1, half = r >> 1;               // A register r = 2 * half + row half
-                            const uint2 o = codes_to_bf16(code[jj][r], zz[hr], sc[hr]);
+                            const uint2 o = kSmallCodes ? small_codes_to_bf16(code[jj][r], cc[hr], sc[hr]) : codes_to_bf16(code[jj][r], zz[hr], sc[hr]);
                             sts64(btile + koff[2 * jj + half] + tl * 2048 + hr * 1024, o.x, o.y);
                         }
                 }

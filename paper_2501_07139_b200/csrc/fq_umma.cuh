@@ -30,13 +30,17 @@ static __device__ __forceinline__ uint32_t g_try_wait(uint32_t bar, uint32_t par
     return ok;
 }
 // Bounded wait; also gives up as soon as another role raised the abort flag.
+//   SLEEP_NS > 0: for waits that last most of a tile (the epilogue's): sleep between polls, leaving the issue slots to the other roles
+template <int SLEEP_NS = 0>
 static __device__ __forceinline__ bool g_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     if (g_try_wait(bar, parity)) return true;
     const unsigned long long t0 = g_ns();
     for (;;) {
-        for (int i = 0; i < 32; i++)
+        for (int i = 0; i < 32; i++) {
             if (g_try_wait(bar, parity)) return true;
+            if constexpr (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
+        }
         if (*abort_flag) return false;
         if (g_ns() - t0 > kGemmWaitNs) return false;
     }
