@@ -380,6 +380,72 @@ def oracle_pass_threads(items, threads):
     return total_bytes, total_s
 
 
+def prefill_oracle_leg(shapes, bits, tokens, n_matrices, rows_per_matrix, device):
+    """The CPU oracle's prefill GEMM on a bounded sample: `rows_per_matrix` sampled token rows of the first
+    `n_matrices` matrices of the prefill stack (all output columns of those rows).  Returns (flop, seconds)."""
+    from oracle import fq_oracle as O
+    flop, secs = 0.0, 0.0
+    for i in range(n_matrices):
+        sh, b = shapes[i], int(bits[i])
+        w = S.weight_rows(S.tensor_key(PREFILL_CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in).numpy()
+        c, sc, z = O.quantize(w, b)
+        x = S.activations(S.tensor_key(PREFILL_CONFIG_ID, sh.k_in, S.TENSOR_X), tokens, sh.k_in, torch.bfloat16, device=device)
+        rows = S.sample_rows(PREFILL_CONFIG_ID * 1000 + i, tokens, rows_per_matrix)[:rows_per_matrix]
+        xb = np.ascontiguousarray(x[torch.from_numpy(rows).to(device)].cpu().view(torch.int16).numpy().view(np.uint16))
+        del x
+        t0 = time.perf_counter()
+        O.gemm(c, sc, z, b, xb)
+        secs += time.perf_counter() - t0
+        flop += 2.0 * len(rows) * sh.n_out * sh.k_in
+    return flop, secs
+
+
+def transition_leg(P, device, blocks=4, high=8, low=4):
+    """Swap-model transitions (Sec. II-C) on `blocks` decoder blocks of the 7B-shaped stack: every matrix has a
+    `high`- and a `low`-bit variant in page-locked host memory; after loading the all-`high` configuration, each
+    step lowers the seven matrices of one block (one module of the chain) with fq_transition_swap: the `low`
+    variants are copied in, then the `high` ones released.  Timed per step with CUDA events."""
+    shapes = S.stack_shapes("7b", blocks)
+    L = len(shapes)
+    tmp = P.FlexQ(L, device.index or 0)
+    fq = P.FlexQ(L, device.index or 0)
+    for i, sh in enumerate(shapes):
+        w = S.weight_rows(S.tensor_key(CONFIG_ID, i, S.TENSOR_W), 0, sh.n_out, sh.k_in, device=device)
+        for b in (high, low):
+            c, sc, z = P.fq_quantize_layer(w, b)
+            store = tmp.fq_pack_layer(i, c, sc, z, b, P.FQ_FMT_PACKED)
+            fq.fq_host_variant(i, sh.n_out, sh.k_in, b, store.cpu().pin_memory())
+        del w, c, sc, z
+    tmp.fq_destroy()
+    torch.cuda.empty_cache()
+    cfg = [high] * L
+    rep0 = fq.fq_transition_swap(cfg)
+    torch.cuda.synchronize()
+    steps = []
+    for blk in range(blocks):
+        for i in range(7 * blk, 7 * blk + 7):
+            cfg[i] = low
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rep = fq.fq_transition_swap(cfg)
+        e1.record()
+        torch.cuda.synchronize()
+        steps.append((e0.elapsed_time(e1), rep))
+    status = fq.fq_status()
+    fq.fq_destroy()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after the transition leg")
+    ms = sorted(t for t, _ in steps)[len(steps) // 2]
+    rep = steps[-1][1]
+    return {"workload": f"{blocks} blocks of the 7B-shaped stack, packed variants of {high} and {low} bits in page-locked host "
+                        f"memory; each step lowers one block's seven matrices {high} -> {low} (fq_transition_swap)",
+            "initial_load_bytes": rep0["bytes_loaded"], "steps": len(steps), "ms_per_step_median": ms,
+            "bytes_loaded_per_step": rep["bytes_loaded"], "bytes_freed_per_step": rep["bytes_freed"],
+            "peak_extra_bytes": rep["peak_extra_bytes"],
+            "granularity_bytes": rep["footprint_from"] - rep["footprint_to"],
+            "h2d_gbs": rep["bytes_loaded"] / (ms * 1e-3) / 1e9}
+
+
 def oracle_desc(n_layers):
     return f"oracle GEMV over the first {n_layers} matrices of the stack ({n_layers / 7:.2g} blocks), single thread"
 
@@ -439,6 +505,7 @@ def main():
     ap.add_argument("--prefill-steps", type=int, default=3)
     ap.add_argument("--prefill-tokens", type=int, default=PREFILL_TOKENS)
     ap.add_argument("--prefill-only", action="store_true", help="run only the prefill leg and print its object")
+    ap.add_argument("--no-transition", action="store_true", help="skip the swap-transition leg")
     ap.add_argument("--no-configs", action="store_true", help="leave the `configs` object (configs 0, 2, 4 in brief) out of the line")
     ap.add_argument("--all-configs", action="store_true",
                     help="instead of the bench line, print one JSON object per other workload (configs 0, 2, 4)")
@@ -603,6 +670,8 @@ def main():
             "two_pass": dict(pf["two_pass"], note="comparison point: dequant_kernel + gemm_kernel (fq_gemm_two_pass)",
                              frac=pf["two_pass"]["tflops"] / sustained),
         }
+    if not args.no_transition and world == 1:
+        line["transition"] = transition_leg(P, device)
     if not args.no_configs and world == 1 and args.blocks == 32:
         line["configs"] = config_report(P, device, 5, brief=True)
     if not args.no_cpu_baseline:
@@ -615,6 +684,15 @@ def main():
                                 "sample": oracle_desc(n_layers).replace("single thread", f"rows of each matrix dealt to {cores} host threads"),
                                 "single_thread": {"value": byts1 / secs1 / 1e9, "unit": UNIT, "cores": 1,
                                                   "sample": oracle_desc(min(7, n_layers))}}
+        if "prefill" in line:
+            pshapes = S.stack_shapes("7b", args.blocks)
+            pbits = S.draw_bits(S.tensor_key(PREFILL_CONFIG_ID, 0, S.TENSOR_BITS), len(pshapes), PREFILL_BITS)
+            pflop, psecs = prefill_oracle_leg(pshapes, pbits, args.prefill_tokens, min(7, len(pshapes)), 16, device)
+            line["prefill"]["cpu_baseline"] = {
+                "value": pflop / psecs / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+                "sample": f"16 sampled token rows of each of the first {min(7, len(pshapes))} matrices, all output columns, "
+                          f"CPU oracle (fp64), single thread",
+                "full_pass_seconds_extrapolated": psecs / pflop * pf["flop_per_pass"]}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

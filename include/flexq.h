@@ -123,6 +123,40 @@ typedef struct fq_transition_report {
 int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
                   fq_transition_report* report_host, void* stream);
 
+/* Swap model of a transition (Sec. II-C: before a block of parameters is swapped out, its replacement has to
+ * be loaded in addition to the current hybrid model; Sec. III-B: one-way moves keep that traffic small).
+ * Only the variants the active configuration uses stay on the device; the others wait in host memory.
+ *
+ * fq_host_variant registers a PACKED variant of `bits` bits of `layer` whose stored bytes (exactly what
+ * fq_pack_layer wrote into a device buffer, fq_store_bytes(n_out, k_in, bits) of them) lie at `store_host`.
+ * The buffer stays the caller's and must outlive the context; page-locked memory makes the copies
+ * asynchronous.  The first variant of a layer fixes its shape.  Nothing is copied here.
+ *
+ * fq_transition_swap moves to configuration `to_bits_host` layer by layer: a layer whose bit-width changes first
+ * gets its new variant (cudaMallocAsync + one cudaMemcpyAsync from the host copy on `stream`, unless it is
+ * resident already), then switches, then releases the variant it used before (cudaFreeAsync on `stream`) if
+ * that one was brought in by an earlier swap and still has its host copy.  Variants given to fq_pack_layer in
+ * the caller's own device buffers are used where they are and never released.  Nested (PLANES) layers only
+ * switch: a child is a prefix of the resident parent.  Decode and prefill calls issued on `stream` afterwards see
+ * the new configuration; calls issued before it keep reading the old variants, which are released in stream order.
+ * The first call (no configuration active yet) loads every layer.
+ * All checks of fq_transition happen before anything changes.  If an allocation or copy fails part-way the call
+ * returns FQ_ERR_CUDA; every layer is then entirely on its old or entirely on its new variant.
+ * Allocates, and may wait for the stream-ordered allocator: a control-path call, not a hot one. */
+typedef struct fq_swap_report {
+    uint64_t bytes_loaded;      /* copied host -> device by this call                              */
+    uint64_t bytes_freed;       /* device memory released by this call                             */
+    uint64_t peak_extra_bytes;  /* most memory held, during the call, beyond what was resident at its start */
+    uint64_t resident_bytes;    /* swapped-in variants on the device after the call                */
+    uint64_t footprint_from;    /* algorithmic footprint (as fq_set_config) before / after         */
+    uint64_t footprint_to;
+    int layers_changed;
+    int one_way;
+} fq_swap_report;
+int fq_host_variant(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, const void* store_host);
+int fq_transition_swap(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
+                       fq_swap_report* report_host, void* stream);
+
 /* The ensemble on disk (Sec. III / V-B: the stored quantized variants whose total size is the paper's
  * "storage cost").  fq_save writes every registered variant of every layer, exactly as stored on the
  * device, plus shapes, formats and the active configuration; it synchronises the device.

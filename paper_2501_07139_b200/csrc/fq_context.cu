@@ -186,6 +186,9 @@ int fq_destroy(fq_ctx* ctx)
         }
         if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
         for (void* p : ctx->owned) cudaFree(p);
+        for (Layer& L : ctx->layers)
+            for (Variant& v : L.var)
+                if (v.swap_owned && v.store) cudaFree(v.store);
     }
     delete ctx;
     return FQ_OK;
@@ -331,6 +334,102 @@ int fq_transition(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int re
     if (require_one_way && !rep.one_way) return FQ_ERR_ONE_WAY;
     const int rc = fq_set_config(ctx, to_bits_host, n_layers, &rep.footprint_to, stream);
     if (rc != FQ_OK) return rc;
+    if (report_host) *report_host = rep;
+    return FQ_OK;
+}
+
+int fq_host_variant(fq_ctx* ctx, int layer, int n_out, int k_in, int bits, const void* store_host)
+{
+    if (!ctx || !store_host) return FQ_ERR_ARG;
+    if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    if (bits < 2 || bits > 8) return FQ_ERR_BITS;
+    if (n_out < 1 || k_in < 1 || k_in % kGroup != 0) return FQ_ERR_SHAPE;
+    if (!aligned(store_host, 16)) return FQ_ERR_ALIGN;
+    Layer& L = ctx->layers[layer];
+    if (L.registered && (L.n_out != n_out || L.k_in != k_in || L.fmt != FQ_FMT_PACKED)) return FQ_ERR_SHAPE;
+    if (!L.registered) {
+        L.registered = true;
+        L.n_out = n_out; L.k_in = k_in; L.fmt = FQ_FMT_PACKED;
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return FQ_ERR_CUDA;
+        ctx->ws_reserved += layer_partial_bytes(n_out, k_in);
+        const int rc = ensure_workspace(ctx, kPartialBase + ctx->ws_reserved + 256);
+        if (rc != FQ_OK) return rc;
+    }
+    L.var[bits].host = store_host;
+    return FQ_OK;
+}
+
+int fq_transition_swap(fq_ctx* ctx, const uint8_t* to_bits_host, int n_layers, int require_one_way,
+                       fq_swap_report* report_host, void* stream)
+{
+    if (!ctx || !to_bits_host) return FQ_ERR_ARG;
+    int registered = 0;
+    for (const Layer& L : ctx->layers) registered += L.registered ? 1 : 0;
+    if (n_layers != registered) return FQ_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    fq_swap_report rep{};
+    rep.one_way = 1;
+    // 1. validate everything: a failing call changes nothing
+    int i = 0;
+    for (const Layer& L : ctx->layers) {
+        if (!L.registered) continue;
+        const int b0 = L.active_bits, b1 = to_bits_host[i++];
+        if (b1 < 2 || b1 > 8) return FQ_ERR_BITS;
+        const Variant& v = L.fmt == FQ_FMT_PLANES ? L.var[8] : L.var[b1];
+        if (!v.present && !(L.fmt == FQ_FMT_PACKED && v.host)) return FQ_ERR_NO_VARIANT;
+        if (b0 != 0 && b1 > b0) rep.one_way = 0;
+        const uint64_t meta = (uint64_t)L.n_out * (uint64_t)(L.k_in / kGroup) * 4u;
+        if (b0 != 0) rep.footprint_from += (uint64_t)L.n_out * (uint64_t)L.k_in * (uint64_t)b0 / 8u + meta;
+        rep.footprint_to += (uint64_t)L.n_out * (uint64_t)L.k_in * (uint64_t)b1 / 8u + meta;
+    }
+    if (require_one_way && !rep.one_way) return FQ_ERR_ONE_WAY;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return FQ_ERR_CUDA;
+    // 2. layer by layer: bring the replacement in, switch, release what it replaced (in that order: the old variant
+    //    serves until the new one is resident, so the extra memory of a step is one variant at a time)
+    i = 0;
+    uint64_t resident_extra = 0;
+    for (Layer& L : ctx->layers) {
+        if (!L.registered) continue;
+        const int b0 = L.active_bits, b1 = to_bits_host[i++];
+        if (b0 == b1) continue;
+        rep.layers_changed++;
+        if (L.fmt == FQ_FMT_PLANES) {                                   // a child is a prefix of what is resident already
+            L.active_bits = b1;
+            continue;
+        }
+        Variant& nv = L.var[b1];
+        const uint64_t nbytes = (uint64_t)store_bytes(L.n_out, L.k_in, b1);
+        if (!nv.present) {
+            void* p = nullptr;
+            if (cudaMallocAsync(&p, nbytes, st) != cudaSuccess) { ctx->config_epoch++; return FQ_ERR_CUDA; }
+            if (cudaMemcpyAsync(p, nv.host, nbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+                cudaFreeAsync(p, st);
+                ctx->config_epoch++;
+                return FQ_ERR_CUDA;
+            }
+            nv.store = p; nv.present = true; nv.swap_owned = true;
+            rep.bytes_loaded += nbytes;
+            resident_extra += nbytes;
+            if (resident_extra > rep.peak_extra_bytes) rep.peak_extra_bytes = resident_extra;
+        }
+        L.active_bits = b1;
+        if (b0 != 0) {
+            Variant& ov = L.var[b0];
+            if (ov.present && ov.swap_owned && ov.host) {               // can be brought back from the host copy
+                const uint64_t obytes = (uint64_t)store_bytes(L.n_out, L.k_in, b0);
+                if (cudaFreeAsync(ov.store, st) != cudaSuccess) { ctx->config_epoch++; return FQ_ERR_CUDA; }
+                ov.store = nullptr; ov.present = false; ov.swap_owned = false;
+                rep.bytes_freed += obytes;
+                resident_extra = resident_extra > obytes ? resident_extra - obytes : 0;
+            }
+        }
+    }
+    ctx->config_epoch++;
+    for (const Layer& L : ctx->layers)
+        for (int b = 2; b <= 8; b++)
+            if (L.registered && L.var[b].present && L.var[b].swap_owned) rep.resident_bytes += (uint64_t)store_bytes(L.n_out, L.k_in, b);
     if (report_host) *report_host = rep;
     return FQ_OK;
 }

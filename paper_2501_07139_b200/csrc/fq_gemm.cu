@@ -307,7 +307,7 @@ int launch_gemm(Ctx* ctx, const void* store, int blob_stride, const FieldList& f
     da.out = static_cast<__nv_bfloat16*>(w_scratch);
     const long long items = (long long)row_tiles(n_out) * supersteps(k_in);     // one warp each
     long long blocks = (items + 7) / 8;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
     dequant_kernel<<<(unsigned)blocks, 256, 0, st>>>(da);
     FQ_CUDA_OK(cudaGetLastError());
 

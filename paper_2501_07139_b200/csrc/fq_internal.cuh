@@ -12,8 +12,10 @@ namespace fq {
 
 // One stored variant of a layer.
 struct Variant {
-    bool present = false;
+    bool present = false;        // resident on the device: kernels may read `store`
     void* store = nullptr;       // blobs: scale/zero words + field arrays (fq_layout.cuh)
+    const void* host = nullptr;  // the same bytes in host memory (swap model, fq_host_variant), or null
+    bool swap_owned = false;     // `store` was allocated by fq_transition_swap: released when the variant is dropped
 };
 
 struct Layer {
@@ -102,6 +104,9 @@ int launch_export_planes(const void* store, int n_out, int k_in, int bits, const
                          uint32_t* out, cudaStream_t st);
 int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, uint16_t* scales, uint16_t* zeros,
                        cudaStream_t st);
+
+// SM count of the current device (cached); sizes the grids of the grid-stride kernels that have no context at hand.
+int current_sm_count();
 
 int launch_stream_read(const void* src, size_t bytes, unsigned* sink, int sm_count, cudaStream_t st);
 

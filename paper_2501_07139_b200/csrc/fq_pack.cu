@@ -78,12 +78,25 @@ quantize_kernel(const float* __restrict__ w, long long n_groups_total, int bits,
     }
 }
 
+int current_sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 132;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 132;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 int launch_quantize(const float* w, int n_out, int k_in, int bits, uint8_t* codes, uint16_t* scales,
                     uint16_t* zeros, cudaStream_t st)
 {
     const long long groups = (long long)n_out * (k_in / kGroup);
     long long blocks = (groups + 7) / 8;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > current_sm_count() * 16) blocks = current_sm_count() * 16;
     if (blocks < 1) return FQ_OK;
     quantize_kernel<<<(unsigned)blocks, 256, 0, st>>>(w, groups, bits, codes, scales, zeros);
     FQ_CUDA_OK(cudaGetLastError());
@@ -151,7 +164,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const StoreArgs a)
 static unsigned grid_for(long long total)
 {
     long long b = (total + 255) / 256;
-    if (b > 148 * 32) b = 148 * 32;
+    if (b > (long long)current_sm_count() * 32) b = (long long)current_sm_count() * 32;
     return (unsigned)(b < 1 ? 1 : b);
 }
 

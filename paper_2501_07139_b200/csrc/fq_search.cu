@@ -12,13 +12,6 @@
 
 namespace {
 
-// One candidate successor of a stem's last configuration.
-struct Cand {
-    int stem, module;          // parent ensemble, module that goes one level down
-    double sens, cost;
-    uint64_t foot;
-};
-
 double state_cost(const uint8_t* st, const double* cost, int M, int Lv)
 {
     double c = 0.0;
@@ -47,6 +40,55 @@ __global__ void sqdiff_kernel(const __nv_bfloat16* a, const __nv_bfloat16* b, si
     if ((threadIdx.x & 31) == 0) { atomicAdd(out, d2); atomicAdd(out + 1, b2); }
 }
 
+// Beam search over one-way precision chains (Sec. III-B, Algorithm 1).  A beam entry is a whole chain
+// (configuration after configuration, M levels each); every round extends each entry by one move, "module m goes
+// down one stored precision", and keeps the `stems` best distinct extensions.
+struct Move { int stem, module; double sens, cost; uint64_t foot; };
+using Chain = std::vector<uint8_t>;
+
+// The moves open to one beam entry, cut down to the `branches` whose single-module sensitivity is smallest
+// (ties keep module order), each scored by the evaluation function of the configuration it leads to.
+void shortlist(int stem, const uint8_t* last, const double* cost, const double* sens, const uint64_t* foot, int M, int Lv,
+               int branches, std::vector<Move>& pool)
+{
+    std::vector<Move> open;
+    for (int m = 0; m < M; m++)
+        if (last[m] + 1 < Lv) open.push_back(Move{stem, m, sens[m * Lv + last[m] + 1], 0.0, 0});
+    std::stable_sort(open.begin(), open.end(), [](const Move& a, const Move& b) { return a.sens < b.sens; });
+    if ((int)open.size() > branches) open.resize(branches);
+    Chain cfg(last, last + M);
+    for (Move& mv : open) {
+        cfg[mv.module]++;
+        mv.cost = state_cost(cfg.data(), cost, M, Lv);
+        mv.foot = state_foot(cfg.data(), foot, M, Lv);
+        cfg[mv.module]--;
+        pool.push_back(mv);
+    }
+}
+
+// The next beam: moves in order of evaluation (then footprint, then beam and module order), each appended to a
+// copy of its entry; a configuration that two entries reach is kept once.
+std::vector<Chain> next_beam(const std::vector<Chain>& beam, std::vector<Move>& pool, int depth, int M, int stems)
+{
+    std::stable_sort(pool.begin(), pool.end(), [](const Move& a, const Move& b) {
+        if (a.cost != b.cost) return a.cost < b.cost;
+        return a.foot < b.foot;
+    });
+    std::vector<Chain> next;
+    for (const Move& mv : pool) {
+        if ((int)next.size() == stems) break;
+        const Chain& from = beam[mv.stem];
+        Chain grown(from.begin(), from.begin() + (size_t)depth * M);
+        grown.insert(grown.end(), from.begin() + (size_t)(depth - 1) * M, from.begin() + (size_t)depth * M);
+        grown[(size_t)depth * M + mv.module]++;
+        bool seen = false;
+        for (const Chain& q : next)
+            if (std::equal(q.end() - M, q.end(), grown.end() - M)) { seen = true; break; }
+        if (!seen) next.push_back(std::move(grown));
+    }
+    return next;
+}
+
 }  // namespace
 
 extern "C" {
@@ -57,58 +99,24 @@ int fq_search_chain(const double* cost, const double* sens, const uint64_t* foot
     if (!cost || !sens || !foot || !chain_out) return FQ_ERR_ARG;
     if (n_modules < 1 || n_levels < 2 || n_levels > 8 || stems < 1 || branches < 1) return FQ_ERR_ARG;
     const int M = n_modules, Lv = n_levels;
-    const int n_steps = M * (Lv - 1);                      // every step lowers one module by one level
-    // an ensemble = the path from QM(n_up) to its last configuration
-    std::vector<std::vector<uint8_t>> paths(1, std::vector<uint8_t>(M, 0));
-    for (int step = 0; step < n_steps; step++) {
-        std::vector<Cand> pool;
-        for (int s = 0; s < (int)paths.size(); s++) {
-            const uint8_t* last = paths[s].data() + (size_t)step * M;
-            // candidateGenerator: one-way successors of this stem's last configuration
-            std::vector<Cand> mine;
-            for (int m = 0; m < M; m++)
-                if (last[m] + 1 < Lv) mine.push_back(Cand{s, m, sens[m * Lv + last[m] + 1], 0.0, 0});
-            // analysisFilter: the #branch least sensitive replacements survive
-            std::stable_sort(mine.begin(), mine.end(), [](const Cand& a, const Cand& b) { return a.sens < b.sens; });
-            if ((int)mine.size() > branches) mine.resize(branches);
-            // calibrationEval
-            for (Cand& c : mine) {
-                std::vector<uint8_t> st(last, last + M);
-                st[c.module]++;
-                c.cost = state_cost(st.data(), cost, M, Lv);
-                c.foot = state_foot(st.data(), foot, M, Lv);
-                pool.push_back(c);
-            }
-        }
-        // rank: lower cost first, then smaller footprint, then stem and module order
-        std::stable_sort(pool.begin(), pool.end(), [](const Cand& a, const Cand& b) {
-            if (a.cost != b.cost) return a.cost < b.cost;
-            return a.foot < b.foot;
-        });
-        std::vector<std::vector<uint8_t>> next;
-        for (const Cand& c : pool) {
-            if ((int)next.size() == stems) break;
-            std::vector<uint8_t> p(paths[c.stem].begin(), paths[c.stem].begin() + (size_t)(step + 1) * M);
-            const std::vector<uint8_t> last(p.end() - M, p.end());
-            p.insert(p.end(), last.begin(), last.end());
-            p[(size_t)(step + 1) * M + c.module]++;
-            bool dup = false;                               // the same configuration reached twice is kept once
-            for (const auto& q : next)
-                if (std::equal(q.end() - M, q.end(), p.end() - M)) { dup = true; break; }
-            if (!dup) next.push_back(std::move(p));
-        }
-        paths.swap(next);
+    const int n_moves = M * (Lv - 1);                       // from all-highest to all-lowest, one level of one module at a time
+    std::vector<Chain> beam(1, Chain(M, 0));
+    for (int depth = 1; depth <= n_moves; depth++) {
+        std::vector<Move> pool;
+        for (int s = 0; s < (int)beam.size(); s++)
+            shortlist(s, beam[s].data() + (size_t)(depth - 1) * M, cost, sens, foot, M, Lv, branches, pool);
+        beam = next_beam(beam, pool, depth, M, stems);
     }
-    // the ensemble with the best trade-off curve: smallest sum of the evaluation over its configurations
+    // the chain whose trade-off curve is best: smallest sum of the evaluation over its configurations
     int best = 0;
     double best_c = 0.0;
-    for (int s = 0; s < (int)paths.size(); s++) {
+    for (int s = 0; s < (int)beam.size(); s++) {
         double c = 0.0;
-        for (int t = 0; t <= n_steps; t++) c += state_cost(paths[s].data() + (size_t)t * M, cost, M, Lv);
+        for (int t = 0; t <= n_moves; t++) c += state_cost(beam[s].data() + (size_t)t * M, cost, M, Lv);
         if (s == 0 || c < best_c) { best = s; best_c = c; }
     }
-    std::copy(paths[best].begin(), paths[best].end(), chain_out);
-    if (n_states_out) *n_states_out = n_steps + 1;
+    std::copy(beam[best].begin(), beam[best].end(), chain_out);
+    if (n_states_out) *n_states_out = n_moves + 1;
     if (curve_cost_out) *curve_cost_out = best_c;
     return FQ_OK;
 }
@@ -159,7 +167,7 @@ int fq_sqdiff(const uint16_t* a_bf16_dev, const uint16_t* b_bf16_dev, size_t n, 
     if (!a_bf16_dev || !b_bf16_dev || !sums_dev || n == 0) return FQ_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(sums_dev, 0, 2 * sizeof(double), st) != cudaSuccess) return FQ_ERR_CUDA;
-    const int blocks = (int)std::min<size_t>((n + 255) / 256, 148 * 8);
+    const int blocks = (int)std::min<size_t>((n + 255) / 256, (size_t)fq::current_sm_count() * 8);
     sqdiff_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(a_bf16_dev),
                                           reinterpret_cast<const __nv_bfloat16*>(b_bf16_dev), n, sums_dev);
     return cudaGetLastError() == cudaSuccess ? FQ_OK : FQ_ERR_CUDA;

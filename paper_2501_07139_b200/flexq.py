@@ -24,12 +24,19 @@ EXPORTS = [
     "fq_set_config", "fq_gemv", "fq_gemv_batched", "fq_gemv_stack", "fq_gemm", "fq_export_layer",
     "fq_export_meta", "fq_storage_bytes", "fq_active_bits", "fq_status", "fq_strerror", "fq_gemv_static", "fq_transition", "fq_save", "fq_load", "fq_search_chain", "fq_prune_chain", "fq_sqdiff",
     "fq_set_wait_limit_ns", "fq_code_bytes", "fq_meta_bytes", "fq_stream_read", "fq_gemm_two_pass",
+    "fq_host_variant", "fq_transition_swap",
 ]
 
 
 class TransitionReport(C.Structure):
     _fields_ = [("bytes_freed", C.c_uint64), ("bytes_loaded", C.c_uint64), ("footprint_from", C.c_uint64),
                 ("footprint_to", C.c_uint64), ("layers_changed", C.c_int), ("one_way", C.c_int)]
+
+
+class SwapReport(C.Structure):
+    _fields_ = [("bytes_loaded", C.c_uint64), ("bytes_freed", C.c_uint64), ("peak_extra_bytes", C.c_uint64),
+                ("resident_bytes", C.c_uint64), ("footprint_from", C.c_uint64), ("footprint_to", C.c_uint64),
+                ("layers_changed", C.c_int), ("one_way", C.c_int)]
 
 
 class FlexQError(RuntimeError):
@@ -60,6 +67,8 @@ def lib():
     L.fq_pack_layer.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
     L.fq_set_config.argtypes = [vp, vp, i, C.POINTER(u64), vp]
     L.fq_transition.argtypes = [vp, vp, i, i, C.POINTER(TransitionReport), vp]
+    L.fq_host_variant.argtypes = [vp, i, i, i, i, vp]
+    L.fq_transition_swap.argtypes = [vp, vp, i, i, C.POINTER(SwapReport), vp]
     L.fq_save.argtypes = [vp, C.c_char_p, C.POINTER(u64)]
     L.fq_load.argtypes = [vp, C.c_char_p]
     L.fq_search_chain.argtypes = [vp, vp, vp, i, i, i, i, vp, C.POINTER(i), C.POINTER(C.c_double)]
@@ -226,6 +235,22 @@ class FlexQ:
         return {"bytes_freed": int(rep.bytes_freed), "bytes_loaded": int(rep.bytes_loaded),
                 "layers_changed": int(rep.layers_changed), "one_way": bool(rep.one_way),
                 "footprint_from": int(rep.footprint_from), "footprint_to": int(rep.footprint_to)}
+
+    def fq_host_variant(self, layer: int, n_out: int, k_in: int, bits: int, store_host: torch.Tensor) -> None:
+        """Registers a PACKED variant whose stored bytes lie in the (page-locked) host tensor `store_host`."""
+        if store_host.device.type != "cpu" or not store_host.is_contiguous():
+            raise ValueError("store_host must be a contiguous host tensor")
+        if store_host.numel() * store_host.element_size() < fq_store_bytes(n_out, k_in, bits, FQ_FMT_PACKED):
+            raise ValueError("store_host is smaller than fq_store_bytes")
+        self._keep[("host", layer, bits)] = store_host       # the library reads it at every swap-in
+        _check(lib().fq_host_variant(self._h, layer, n_out, k_in, bits, store_host.data_ptr()), "fq_host_variant")
+
+    def fq_transition_swap(self, bits: Sequence[int], require_one_way: bool = True) -> dict:
+        arr = (C.c_uint8 * len(bits))(*[int(b) for b in bits])
+        rep = SwapReport()
+        _check(lib().fq_transition_swap(self._h, arr, len(bits), 1 if require_one_way else 0, C.byref(rep), _stream()),
+               "fq_transition_swap")
+        return {k: int(getattr(rep, k)) for k, _ in SwapReport._fields_}
 
     def fq_save(self, path: str) -> int:
         """Writes every stored variant to `path`; returns the bytes written."""

@@ -4,7 +4,9 @@ library's tree search (Sec. III-B, Algorithm 1) and pruning (Sec. III-C) on them
 The paper evaluates candidates by perplexity on a calibration set; without trained weights and datasets the
 evaluation here is the relative output error of each linear layer on seeded calibration activations,
 || Y_b - Y_8 ||^2 / || Y_8 ||^2, summed over the layers of a module (and over modules for a configuration).
-All arithmetic runs in the library: fq_gemm for the outputs, fq_sqdiff for the error sums."""
+The library does the heavy work: fq_gemm for the outputs, fq_sqdiff for the two fp64 sums of every comparison,
+fq_code_bytes for the sizes, fq_search_chain / fq_prune_chain for the search.  This module only divides each pair
+of sums and adds the per-layer ratios and sizes up per module (a few hundred host operations)."""
 from __future__ import annotations
 
 from typing import Dict, List, Sequence
@@ -51,7 +53,7 @@ def module_tables(fq: "F.FlexQ", shapes: Sequence, modules: Sequence[Sequence[in
 
     cost = [[sum(rel(err[i][li]) for i in mod) for li in range(n_lev)] for mod in modules]
     sens = [[sum(rel(err_s[i][li]) for i in mod) for li in range(n_lev)] for mod in modules]
-    foot = [[sum(shapes[i].n_out * shapes[i].k_in * int(b) // 8 for i in mod) for b in levels] for mod in modules]
+    foot = [[sum(F.fq_code_bytes(shapes[i].n_out, shapes[i].k_in, int(b)) for i in mod) for b in levels] for mod in modules]
     return cost, sens, foot
 
 

@@ -49,3 +49,89 @@ def test_transition_reports_match_oracle_and_respect_one_way():
     ref = O.gemv(q8c[0] >> 3, q8c[1], q8c[2], 5, bits_of(x), parent_bits=8)[0]
     assert O.rel_l2(f64_of(y), ref) <= GEMV_TOL and fq.fq_status() == 0
     fq.fq_destroy()
+
+
+def test_swap_transition_loads_before_it_releases_and_decodes_bit_identically():
+    """Swap model (Sec. II-C): only the active variants are on the device, the others wait in page-locked host
+    memory; a one-way chain of swaps against a context that keeps everything resident."""
+    import fq_synth as S
+    import paper_2501_07139_b200 as P
+    dev = torch.device("cuda", 0)
+    shapes = [(2048, 4096), (1000, 2048), (4096, 1024)]
+    variants = (8, 5, 3)
+    ref = P.FlexQ(4)                                       # everything resident
+    fq = P.FlexQ(4)                                        # swap model
+    sizes = {}
+    for i, (n, k) in enumerate(shapes):
+        w = S.weight_rows(S.tensor_key(140, i, S.TENSOR_W), 0, n, k, device=dev)
+        for b in variants:
+            c, s, z = P.fq_quantize_layer(w, b)
+            store = ref.fq_pack_layer(i, c, s, z, b, P.FQ_FMT_PACKED)
+            sizes[(i, b)] = store.numel()
+            assert store.numel() == P.fq_store_bytes(n, k, b, P.FQ_FMT_PACKED)
+            fq.fq_host_variant(i, n, k, b, store.cpu().pin_memory())
+    # layer 3: a nested parent, resident in both
+    w = S.weight_rows(S.tensor_key(140, 3, S.TENSOR_W), 0, 512, 1024, device=dev)
+    c, s, z = P.fq_quantize_layer(w, 8)
+    ref.fq_pack_layer(3, c, s, z, 8, P.FQ_FMT_PLANES)
+    fq.fq_pack_layer(3, c, s, z, 8, P.FQ_FMT_PLANES)
+    all_shapes = shapes + [(512, 1024)]
+    xs = [S.activations(S.tensor_key(140, i, S.TENSOR_X), 1, k).to(dev)[0] for i, (n, k) in enumerate(all_shapes)]
+
+    def same_outputs(cfg):
+        ref.fq_set_config(cfg)
+        for i, (n, k) in enumerate(all_shapes):
+            ya = torch.full((n,), float("nan"), dtype=torch.float16, device=dev)
+            yb = torch.full((n,), float("nan"), dtype=torch.float16, device=dev)
+            ref.fq_gemv(i, xs[i], ya)
+            fq.fq_gemv(i, xs[i], yb)
+            assert torch.equal(ya, yb), (cfg, i)
+        ys = [torch.empty(n, dtype=torch.float16, device=dev) for n, _ in all_shapes]
+        yr = [torch.empty(n, dtype=torch.float16, device=dev) for n, _ in all_shapes]
+        fq.fq_gemv_stack(list(range(4)), xs, ys, None, 1)
+        ref.fq_gemv_stack(list(range(4)), xs, yr, None, 1)
+        assert all(torch.equal(a, b) for a, b in zip(ys, yr))
+        assert fq.fq_status() == 0 and ref.fq_status() == 0
+
+    n_all, k_all = [s[0] for s in all_shapes], [s[1] for s in all_shapes]
+    # nothing usable before the first swap: the packed layers have no resident variant
+    with pytest.raises(P.FlexQError):
+        fq.fq_set_config([8, 8, 8, 8])
+    cur = [8, 8, 8, 8]
+    rep = fq.fq_transition_swap(cur)
+    assert rep["bytes_loaded"] == sum(sizes[(i, 8)] for i in range(3)) and rep["bytes_freed"] == 0
+    assert rep["resident_bytes"] == rep["bytes_loaded"] and rep["footprint_to"] == O.footprint(n_all, k_all, cur)
+    same_outputs(cur)
+    resident = rep["resident_bytes"]
+    for nxt in ([8, 5, 8, 6], [3, 5, 8, 6], [3, 3, 5, 4], [3, 3, 3, 2]):
+        torch.cuda.synchronize()
+        free0 = torch.cuda.mem_get_info()[0]
+        rep = fq.fq_transition_swap(nxt)
+        changed = [i for i in range(3) if cur[i] != nxt[i]]
+        loaded = sum(sizes[(i, nxt[i])] for i in changed)
+        freed = sum(sizes[(i, cur[i])] for i in changed)
+        assert rep["bytes_loaded"] == loaded and rep["bytes_freed"] == freed and rep["one_way"] == 1
+        assert rep["layers_changed"] == sum(1 for a, b in zip(cur, nxt) if a != b)
+        # a layer's replacement is resident before the layer's old variant goes, one layer at a time
+        assert rep["peak_extra_bytes"] == max(sizes[(i, nxt[i])] for i in changed)
+        resident += loaded - freed
+        assert rep["resident_bytes"] == resident
+        assert rep["footprint_from"] == O.footprint(n_all, k_all, cur) and rep["footprint_to"] == O.footprint(n_all, k_all, nxt)
+        torch.cuda.synchronize()
+        free1 = torch.cuda.mem_get_info()[0]
+        assert free1 - free0 >= (freed - loaded) - (8 << 20)          # the memory really went back (pool granularity aside)
+        cur = nxt
+        same_outputs(cur)
+    # one-way is enforced before anything moves; a width that was never registered is refused
+    with pytest.raises(P.FlexQError) as e:
+        fq.fq_transition_swap([5, 3, 3, 2])
+    assert e.value.code == -10 and [fq.fq_active_bits(i) for i in range(4)] == cur
+    with pytest.raises(P.FlexQError) as e:
+        fq.fq_transition_swap([3, 3, 2, 2])
+    assert e.value.code == -5 and [fq.fq_active_bits(i) for i in range(4)] == cur
+    # going back up is a swap like any other when the caller allows it
+    rep = fq.fq_transition_swap([8, 3, 3, 7], require_one_way=False)
+    assert rep["one_way"] == 0 and rep["bytes_loaded"] == sizes[(0, 8)] and rep["bytes_freed"] == sizes[(0, 3)]
+    same_outputs([8, 3, 3, 7])
+    fq.fq_destroy()
+    ref.fq_destroy()
