@@ -49,7 +49,9 @@ enum { FQ_OK = 0,
        FQ_ERR_TIMEOUT = -8,     /* a bounded device-side wait ran out (see fq_status)       */
        FQ_ERR_SCRATCH = -9,     /* problem needs more than the built-in scratch (fq_gemv_static) */
        FQ_ERR_ONE_WAY = -10,    /* a layer would go to a higher bit-width (fq_transition)    */
-       FQ_ERR_IO = -11 };       /* file could not be opened, read or written, or is malformed */
+       FQ_ERR_IO = -11,         /* file could not be opened, read or written, or is malformed */
+       FQ_ERR_BOUNDS = -12 };   /* checked build only (-DFQ_CHECKED): a kernel computed an address outside its
+                                   buffer; the access was skipped (see fq_status)                         */
 
 #define FQ_MAX_BATCH 8          /* decode batch handled by the GEMV family */
 

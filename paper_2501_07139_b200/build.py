@@ -9,6 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libflexq.so")
+LIB_CHECKED = os.path.join(HERE, "libflexq_checked.so")     # the same sources with -DFQ_CHECKED (bounds-checked kernels)
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -20,26 +21,30 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + \
         glob.glob(os.path.join(HERE, "..", "include", "*.h")) + [os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compiles every .cu under csrc/ into libflexq.so next to this file (if stale)."""
-    if not force and not _stale():
-        return LIB
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compiles every .cu under csrc/ into libflexq.so next to this file (if stale).  checked=True builds
+    libflexq_checked.so instead: the kernels verify every global-memory index they compute against the size of
+    the buffer it falls in, skip an access that would be outside and report FQ_ERR_BOUNDS through fq_status."""
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + sources()
+    tmp = lib + f".tmp{os.getpid()}"
+    cmd = [nvcc] + NVCC_FLAGS + (["-DFQ_CHECKED"] if checked else []) + (["-Xptxas", "-v"] if verbose else []) + \
+        ["-o", tmp] + sources()
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

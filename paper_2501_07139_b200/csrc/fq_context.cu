@@ -142,6 +142,7 @@ const char* fq_strerror(int code)
         case FQ_ERR_SCRATCH: return "layer needs more than the built-in scratch";
         case FQ_ERR_ONE_WAY: return "transition would raise a layer's bit-width";
         case FQ_ERR_IO: return "file could not be opened, read or written, or is malformed";
+        case FQ_ERR_BOUNDS: return "a kernel computed an address outside its buffer (checked build)";
         default: return "unknown error";
     }
 }

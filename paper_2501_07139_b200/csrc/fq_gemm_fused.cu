@@ -346,6 +346,11 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                 // ---- the stored words of this stage (64 columns = k32 steps j0, j0 + 1 of one superstep of one blob)
                 const int kb = ks >> 3, ssl = (ks >> 2) & 1, j0 = (ks & 3) * 2, grp = (ks >> 1) & 1;
                 const uint8_t* blob_lane = row_blobs + (long long)kb * a.blob_stride;
+                if (!FQ_IN_BOUNDS(kb < a.n_kb && (have ? rp : 0) < n_rp && stage < kFStages, a.status)) {   // (checked build)
+                    if (lane == 0) *abort_flag = 1;
+                    ok = false;
+                    break;
+                }
                 uint4 raw[kBlobTiles][kLoads];
                 uint2 meta[kBlobTiles];                                    // scale / zero words of rows g and g + 8: adjacent
                 load_stage_words<VARIANT, 0>(blob_lane, ssl, j0, raw[0]);

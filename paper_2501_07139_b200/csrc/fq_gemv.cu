@@ -566,6 +566,14 @@ gemv_kernel(const __grid_constant__ GemvOp single, const StackArgs sa)
                         ok = __shfl_sync(0xffffffffu, ok, 0);
                         if (!ok) { stop = true; break; }
                         const uint32_t stage_base = smem_u32(smem + S::oStages) + (uint32_t)stage * S::kStageBytes;
+                        // (checked build) the blobs of this copy lie inside the stored variant and fit the stage; the
+                        // transaction stays pending, the status word ends every wait
+                        if (!FQ_IN_BOUNDS(rp >= 0 && rp < n_rp && kb0 >= 0 && kb0 + nb <= n_kb && bytes <= (uint32_t)S::kStageBytes,
+                                          sa.status)) {
+                            if (lane == 0) { flags[0] = 1; flags[1] = 1; }
+                            stop = true;
+                            break;
+                        }
                         if (contiguous) {
                             if (lane == 0) bulk_g2s(stage_base, src, bytes, full);
                         } else if (lane < nb) {

@@ -405,6 +405,13 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                     const int nb = min(cb, kb_hi - kb);
                     const uint32_t full = bars + 8 * stage, empty = bars + 128 + 8 * stage;
                     const uint32_t stage_base = sbase + S::oStages + (uint32_t)stage * kStageBytes;
+                    // (checked build) the blobs of this copy lie inside the stored variant and fit the stage
+                    if (!FQ_IN_BOUNDS(rp >= 0 && rp < row_pairs(n_out) && kb >= 0 && kb + nb <= n_kb &&
+                                      (uint32_t)nb * blob_read <= (uint32_t)kStageBytes && sslot < kStripSlots, a.status)) {
+                        if (lane == 0) ctl[S::cAbort] = 1u;
+                        stop = true;
+                        break;
+                    }
                     int ok = 1;
                     if (lane == 0) {
                         if (wraps > 0 && !wait_mbar(empty, (wraps - 1u) & 1u, ctl, a.wait_ns)) {
@@ -538,8 +545,8 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             r0 = r1 = make_uint4(0u, 0u, 0u, 0u);
             const int k = it.kb * 512 + lane * 8;
             if (it.uses > 0) {
-                if (k < it.k_in) r0 = ldg128_hint(it.x + k, keep_policy);
-                if (k + 256 < it.k_in) r1 = ldg128_hint(it.x + k + 256, keep_policy);
+                if (k < it.k_in && FQ_IN_BOUNDS(k + 8 <= it.k_in, a.status)) r0 = ldg128_hint(it.x + k, keep_policy);
+                if (k + 256 < it.k_in && FQ_IN_BOUNDS(k + 264 <= it.k_in, a.status)) r1 = ldg128_hint(it.x + k + 256, keep_policy);
             }
         };
         // Converts a blob into its slot and publishes it.  False: a wait ran out.
@@ -655,8 +662,10 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             {
                 const float v = c == 0 ? tot[0][0] : c == 1 ? tot[0][1] : c == 2 ? tot[1][0] : tot[1][1];
                 const int lr = (c >> 1) * kTileRows + g + 8 * (c & 1);
-                if (finish) part[(sslot * kMaxKb + kb) * 32 + lr] = v;
-                else st_relaxed_u64(dpart + kb * 32 + lr, tag | __float_as_uint(v));   // finished elsewhere
+                if (FQ_IN_BOUNDS(kb >= 0 && kb < d.n_kb && kb < kMaxKb && sslot >= 0 && sslot < kStripSlots, a.status)) {
+                    if (finish) part[(sslot * kMaxKb + kb) * 32 + lr] = v;
+                    else st_relaxed_u64(dpart + kb * 32 + lr, tag | __float_as_uint(v));   // finished elsewhere
+                }
             }
             __threadfence_block();
             __syncwarp();
@@ -705,7 +714,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                 }
                 if (live) {
                     const int row = d.row_base + lane;
-                    if (row < d.n_out) reinterpret_cast<__half*>(d.y)[row] = __float2half_rn(sum);
+                    if (row < d.n_out && FQ_IN_BOUNDS(row >= 0, a.status)) reinterpret_cast<__half*>(d.y)[row] = __float2half_rn(sum);
                 }
             }
             const int phase = d.phase;
@@ -723,7 +732,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                     const unsigned done = atomicAdd(const_cast<unsigned*>(&ctl[S::cFinCnt + (phase & 7)]), 1u) + 1u;
                     if (done == (unsigned)fin_total[phase]) {
                         ctl[S::cFinCnt + (phase & 7)] = 0u;
-                        red_add_relaxed_u64(a.phase_done + phase, 1ull);
+                        if (FQ_IN_BOUNDS(phase < a.n_phases, a.status)) red_add_relaxed_u64(a.phase_done + phase, 1ull);
                     }
                 }
             }

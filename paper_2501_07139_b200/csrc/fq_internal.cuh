@@ -105,6 +105,17 @@ int launch_export_planes(const void* store, int n_out, int k_in, int bits, const
 int launch_export_meta(const void* store, int n_out, int k_in, int stored_bits, uint16_t* scales, uint16_t* zeros,
                        cudaStream_t st);
 
+// Checked build (-DFQ_CHECKED): `inside` states that an index a kernel computed lies inside the buffer it is about to
+// touch.  When it does not hold, the status word gets FQ_ERR_BOUNDS (the first error wins) and the result is false:
+// the caller skips the access and winds the kernel down the way it does after a timeout.  Every lane of the
+// warp evaluates the same condition wherever the result steers control flow.  In the normal build the condition
+// is not evaluated.
+#ifdef FQ_CHECKED
+#define FQ_IN_BOUNDS(inside, status_ptr) ((inside) ? true : (atomicCAS((status_ptr), 0, FQ_ERR_BOUNDS), false))
+#else
+#define FQ_IN_BOUNDS(inside, status_ptr) true
+#endif
+
 // SM count of the current device (cached); sizes the grids of the grid-stride kernels that have no context at hand.
 int current_sm_count();
 

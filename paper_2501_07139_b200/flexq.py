@@ -16,7 +16,11 @@ FQ_FMT_PLANES = 1
 FQ_MAX_BATCH = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libflexq.so")
+# FLEXQ_LIBRARY selects the file: unset = libflexq.so, "checked" = libflexq_checked.so (the bounds-checked build,
+# `python -m paper_2501_07139_b200.build --checked`), anything else = a path.
+_LIB_PATH = {None: os.path.join(_HERE, "libflexq.so"), "": os.path.join(_HERE, "libflexq.so"),
+             "checked": os.path.join(_HERE, "libflexq_checked.so")}.get(os.environ.get("FLEXQ_LIBRARY"),
+                                                                        os.environ.get("FLEXQ_LIBRARY"))
 _lib = None
 
 EXPORTS = [
