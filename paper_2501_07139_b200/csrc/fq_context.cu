@@ -603,6 +603,26 @@ int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_de
     return launch_gemv_static(ctx, op, op_partial_bytes(op, 1), (cudaStream_t)stream);
 }
 
+// Relative cost of a byte, x64, per variant (0..6 packed 2..8 bits, 7..13 nested 2..8 bits).
+static unsigned deal_weight(int variant)
+{
+    static const unsigned w[kVariants] = {125, 112, 66, 78, 78, 84, 48,        // packed 2..8
+                                          133, 107, 103, 114, 127, 124, 120};  // nested 2..8
+    return variant >= 0 && variant < kVariants ? w[variant] : 64u;
+}
+
+// Time a CTA spends on one blob of an op, in arbitrary units: bytes x the relative cost of a byte of the op's
+// variant.  The 8-bit and 4-bit loops keep up with the CTA's share of HBM; variants with more fields per stored
+// bit are bound by the integer pipe and take longer per byte (per-CTA rates of uniform stacks, all CTAs busy:
+// 8 bits 48.8 GB/s, 4: 46.1, 5: 42.8, 6: 42.5, 7: 39.9, 3: 31.5, 2: 27.7; nested children 27 - 34).  The table
+// starts from the inverse rates; the 8-bit entry is lower than that because a CTA that streams 8-bit blobs speeds
+// up when its neighbours are compute-bound and leave it more of the HBM (tuned on the mixed 7B stack: the
+// unordered pass went from 4350 to 5380 GB/s, the ordered one from 1.525 to 1.465 ms).
+static unsigned long long blob_cost(const GemvOp& op)
+{
+    return (unsigned long long)(unsigned)op.blob_read * deal_weight(op.variant);
+}
+
 int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t* const* x_dev_host,
                   uint16_t* const* y_dev_host, const int* phases_host, int batch, void* stream)
 {
@@ -681,9 +701,10 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
             for (int p = 0; p < np; p++) phase_total[p] = 0;
             // ... and for every (CTA, op) the strips the CTA computes.  The ops of one dependency phase (of the
             // whole list when there are no phases) are dealt together: their blobs form one sequence, op
-            // after op, and every CTA gets the same number of BYTES of it in one contiguous piece.  A CTA
-            // then touches one or two ops of a phase instead of all of them: fewer activation vectors to
-            // convert, fewer strips shared with a neighbour.
+            // after op, and every CTA gets the same amount of WORK of it in one contiguous piece (bytes weighted by
+            // what a byte of the op's variant costs a CTA, blob_cost()).  A CTA then touches one or two ops of a
+            // phase instead of all of them: fewer activation vectors to convert, fewer strips shared with a
+            // neighbour.
             uint2* ranges = reinterpret_cast<uint2*>(host + range_off);
             std::vector<int> last_phase(grid, -1);
             for (int g0 = 0, group = 0; g0 < n_ops; group++) {
@@ -692,7 +713,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
                 unsigned long long total = 0;
                 long long strips = 0;
                 for (int i = g0; i < g1; i++) {
-                    total += (unsigned long long)ops[i].n_units * (unsigned)ops[i].blob_read;
+                    total += (unsigned long long)ops[i].n_units * blob_cost(ops[i]);
                     strips += ops[i].n_rp;
                 }
                 // A group with few strips per CTA is dealt in whole strips: such a phase is short, and what
@@ -702,7 +723,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
                 const int rot = (int)((unsigned)group * 53u % (unsigned)grid);      // spreads the remainders
                 unsigned long long before = 0;
                 for (int i = g0; i < g1; i++) {
-                    const unsigned long long sz = (unsigned)ops[i].blob_read;
+                    const unsigned long long sz = blob_cost(ops[i]);
                     const unsigned long long bytes = (unsigned long long)ops[i].n_units * sz;
                     const unsigned long long strip_bytes = (unsigned long long)ops[i].n_kb * sz;
                     for (int c = 0; c < grid; c++) {
