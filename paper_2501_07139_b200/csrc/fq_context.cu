@@ -40,6 +40,15 @@ const Variant* active_variant(const Layer& L, int bits)
     return v.present ? &v : nullptr;
 }
 
+// Batch 1: a group of ops (one dependency phase) that gives a CTA fewer blobs than this is cut into items of one
+// 16-row tile instead of one blob, so that its 16 consumer warps end the phase after the same number of items
+// (a phase of the 7B stack is 7 to 37 blobs per CTA: whole blobs leave the phase waiting for 1, 2 or 3 blob times
+// where half blobs need 0.5, 1.5 or 2.5).  Long groups keep whole blobs, and so do variants of one or two fields,
+// whose blobs are cheap: an item has fixed costs (measured on the 7B stack, ordered: nested 7-bit 2.66 -> 2.36 ms
+// with half blobs, packed mixed 1.46 -> 1.55 ms, so only the many-field variants are cut).
+constexpr int kSplitBelowBlobsPerCta = 48;
+constexpr int kSplitAboveFields = 2;
+
 // Fills the device descriptor of one decode op (everything except workspace pointers and unit_base).
 int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch, GemvOp& op)
 {
@@ -82,6 +91,8 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     if (batch == 1 && L.k_in > gemv1_max_k()) return FQ_ERR_SHAPE;                   // a strip's activations stay in shared memory
     op.phase = -1;
     op.rot = 0;
+    // a lone matrix is a few blobs per CTA: items of one 16-row tile spread them over twice as many consumer warps
+    op.split = (batch == 1 && fl.n > kSplitAboveFields && op.n_units < kSplitBelowBlobsPerCta * ctx->sm_count) ? 2 : 1;
     return FQ_OK;
 }
 
@@ -716,6 +727,10 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
                     total += (unsigned long long)ops[i].n_units * blob_cost(ops[i]);
                     strips += ops[i].n_rp;
                 }
+                long long group_blobs = 0;
+                for (int i = g0; i < g1; i++) group_blobs += ops[i].n_units;
+                for (int i = g0; i < g1; i++)
+                    ops[i].split = (ops[i].n_fields > kSplitAboveFields && group_blobs < (long long)kSplitBelowBlobsPerCta * grid) ? 2 : 1;
                 // A group with few strips per CTA is dealt in whole strips: such a phase is short, and what
                 // counts is that no CTA has to wait for a neighbour's share of a strip, not the last few
                 // per cent of balance.

@@ -58,10 +58,10 @@ constexpr int kMaxOpsDev = 512;                        // ops of one launch (the
 // What the producer tells a consumer warp about one item (one 16-byte store, one 16-byte load).
 //   w0 blob shared address   w1 packed fields (below)   w2 activation blob number + 1   w3 sequence tag
 constexpr uint32_t kItemEnd = 1u << 31;
-__device__ __forceinline__ uint32_t item_pack(int xslot, int stage, int parity, int kb, int sslot, int variant)
+__device__ __forceinline__ uint32_t item_pack(int xslot, int stage, int parity, int kb, int sslot, int variant, int tsel)
 {
     return (uint32_t)xslot | (uint32_t)stage << 5 | (uint32_t)parity << 9 | (uint32_t)kb << 10 | (uint32_t)sslot << 15 |
-           (uint32_t)variant << 18;
+           (uint32_t)variant << 18 | (uint32_t)tsel << 22;
 }
 
 // A strip in flight.
@@ -351,13 +351,14 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             const uint8_t* store;
             unsigned long long* partial;
             uint16_t* y;
-            int blob_read, blob_stride, n_kb, cb, variant, n_out, phase;
+            int blob_read, blob_stride, n_kb, cb, variant, n_out, phase, split;
             __device__ __forceinline__ void fetch(const GemvOp* ops, int oi, int n_ops)
             {
                 if (oi >= n_ops) return;
                 const GemvOp& o = ops[oi];
                 store = o.store; partial = o.partial; y = o.y; blob_read = o.blob_read; blob_stride = o.blob_stride;
                 n_kb = o.n_kb; cb = o.chunk_blobs; variant = o.variant; n_out = o.n_out; phase = o.phase;
+                split = o.split == 2 ? 2 : 1;
             }
         };
         OpRegs nxt;
@@ -366,6 +367,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             const OpRegs cur = nxt;
             nxt.fetch(ops, oi + 1, a.n_ops);
             const int n_kb = cur.n_kb, cb = cur.cb, variant = cur.variant, n_out = cur.n_out, phase = cur.phase;
+            const int split = cur.split;                 // items per blob: the whole blob, or one 16-row tile each
             const StripOrder so(range[oi], n_kb);
             if (so.n_strips == 0) continue;
             const uint32_t blob_read = (uint32_t)cur.blob_read;
@@ -394,7 +396,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                     if (lane == 0) d = make_uint4((uint32_t)(uintptr_t)y, (uint32_t)((uintptr_t)y >> 32), (uint32_t)(uintptr_t)sp,
                                                   (uint32_t)((uintptr_t)sp >> 32));
                     else if (lane == 1) d = make_uint4((uint32_t)n_out, (uint32_t)(rp * (kBlobTiles * kTileRows)), (uint32_t)n_kb, (uint32_t)kb_lo);
-                    else d = make_uint4((uint32_t)kb_hi, c0 == 0 ? 1u : 0u, (uint32_t)phase, (uint32_t)(kb_hi - kb_lo));
+                    else d = make_uint4((uint32_t)kb_hi, c0 == 0 ? 1u : 0u, (uint32_t)phase, (uint32_t)((kb_hi - kb_lo) * split));
                     if (lane < 3) sts128(sdesc_a + (uint32_t)sslot * 64u + (uint32_t)lane * 16u, d);
                     if (lane == 0) ctl[S::cStripBusy + sslot] = 1u;
                     __threadfence_block();                           // the descriptor before any item that refers to it
@@ -421,25 +423,28 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                         if (ok) {
                             mbar_expect_tx(full, (uint32_t)nb * blob_read);
                             if (contiguous) bulk_g2s_hint(stage_base, src, (uint32_t)nb * blob_read, full, stream_policy);
-                            mbar_arrive_n(empty, (uint32_t)(kCW - nb));   // for the warps without an item in this unit
+                            mbar_arrive_n(empty, (uint32_t)(kCW - nb * split));   // for the warps without an item in this unit
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) { stop = true; break; }
                     if (!contiguous && lane < nb) bulk_g2s_hint(stage_base + lane * blob_read, src + lane * blob_stride, blob_read, full, stream_policy);
-                    // the items of this unit: blob b goes to consumer warp (rr + b) mod 16
-                    const int b = (int)((unsigned)my_klane - rr) & (kKLanes - 1);
-                    if (lane < kCW && b < nb) {
+                    // the items of this unit: item i goes to consumer warp (rr + i) mod 16; item i is blob i, or tile
+                    // i % 2 of blob i / 2
+                    const int item = (int)((unsigned)my_klane - rr) & (kKLanes - 1);
+                    if (lane < kCW && item < nb * split) {
+                        const int b = split == 2 ? item >> 1 : item;
+                        const int tsel = split == 2 ? 1 + (item & 1) : 0;
                         const unsigned xs = xseq + (unsigned)(kb + b);
                         uint4 e;
                         e.x = stage_base + (uint32_t)b * blob_read;
-                        e.y = item_pack((int)(xs % kXSlots), stage, (int)(wraps & 1u), kb + b, sslot, variant);
+                        e.y = item_pack((int)(xs % kXSlots), stage, (int)(wraps & 1u), kb + b, sslot, variant, tsel);
                         e.z = xs + 1u;
                         e.w = qn + 1u;
                         sts128(my_queue + (qn % kQD) * 16u, e);
                         qn++;
                     }
-                    rr += (unsigned)nb;
+                    rr += (unsigned)(nb * split);
                     src += (long long)nb * blob_stride;
                     if (++stage == S::kStages) { stage = 0; wraps++; }
                 }
@@ -474,13 +479,14 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
         };
         // iterator over this warp's blobs
         int it_oi = -1, it_kb = 0, it_nkb = 0, it_kin = 0, it_phase = -1;
-        int fk0 = 0, fk1 = 0, lk0 = 0, lk1 = 0, n_mid = 0, two = 0;
+        int fk0 = 0, fk1 = 0, lk0 = 0, lk1 = 0, n_mid = 0, two = 0, it_split = 1;
         unsigned xbase = 0;
         const __half* it_x = nullptr;
         auto advance = [&](Item& it) -> bool {
             for (;;) {
                 if (it_kb < it_nkb) {
                     int uses = n_mid + ((it_kb >= fk0 && it_kb < fk1) ? 1 : 0) + ((two && it_kb >= lk0 && it_kb < lk1) ? 1 : 0);
+                    uses *= it_split;                                // items, not blobs, count down the slot
                     it.x = it_x; it.k_in = it_kin; it.kb = it_kb; it.uses = uses; it.phase = it_phase;
                     it.xs = xbase + (unsigned)it_kb;
                     it_kb += kPrepWarps;
@@ -493,7 +499,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
                 prefetch_ops(ops, it_oi, a.n_ops, lane);
                 const GemvOp& op = ops[it_oi];
                 const StripOrder so(range[it_oi], op.n_kb);
-                it_nkb = op.n_kb; it_kin = op.k_in; it_phase = op.phase;
+                it_nkb = op.n_kb; it_kin = op.k_in; it_phase = op.phase; it_split = op.split == 2 ? 2 : 1;
                 it_x = reinterpret_cast<const __half*>(op.x);
                 // blobs of x that this CTA's strips cover: the first and the last strip may be partial
                 int f0, f1, l0, l1;
@@ -625,6 +631,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             if (e.y & kItemEnd) break;
             const int xslot = (int)(e.y & 31u), stage = (int)((e.y >> 5) & 15u), parity = (int)((e.y >> 9) & 1u);
             const int kb = (int)((e.y >> 10) & 31u), sslot = (int)((e.y >> 15) & 7u), variant = (int)((e.y >> 18) & 15u);
+            const int tsel = (int)((e.y >> 22) & 3u);                        // 0: both tiles, 1 / 2: tile 0 / 1 only
             // ---- its weights and its activations
             bool ok = wait_mbar(bars + 8 * stage, (uint32_t)parity, ctl, a.wait_ns);
             // (a hardware wake-up: at the start of a dependency phase every consumer sleeps here and must not
@@ -641,7 +648,7 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             for (int jc = 0; jc < 4; jc++)
                 xd[jc] = (g >> 1) == jc ? xdig + x_digit_off(0, jc, g & 1, c) : sbase + S::oZero + c * 16;
             float tot[kBlobTiles][2] = {{0.f, 0.f}, {0.f, 0.f}};
-            blob_dispatch(variant, e.x, xd, sbase + S::oXGrp + (uint32_t)xslot * kXBlobGroupBytes, lane, tot);
+            blob_dispatch(variant, e.x, xd, sbase + S::oXGrp + (uint32_t)xslot * kXBlobGroupBytes, lane, tsel, tot);
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(bars + 128 + 8 * stage);                         // the stage may be refilled
@@ -662,7 +669,8 @@ gemv1_kernel(const __grid_constant__ GemvOp single, const Args a)
             {
                 const float v = c == 0 ? tot[0][0] : c == 1 ? tot[0][1] : c == 2 ? tot[1][0] : tot[1][1];
                 const int lr = (c >> 1) * kTileRows + g + 8 * (c & 1);
-                if (FQ_IN_BOUNDS(kb >= 0 && kb < d.n_kb && kb < kMaxKb && sslot >= 0 && sslot < kStripSlots, a.status)) {
+                if ((tsel == 0 || (c >> 1) == tsel - 1) &&                    // (rows of the tile(s) this item computed)
+                    FQ_IN_BOUNDS(kb >= 0 && kb < d.n_kb && kb < kMaxKb && sslot >= 0 && sslot < kStripSlots, a.status)) {
                     if (finish) part[(sslot * kMaxKb + kb) * 32 + lr] = v;
                     else st_relaxed_u64(dpart + kb * 32 + lr, tag | __float_as_uint(v));   // finished elsewhere
                 }

@@ -190,8 +190,10 @@ __device__ __forceinline__ void group_epilogue(const uint4 mw, const int (&v)[2]
 // bodies would not fit the instruction cache.
 //   blob : shared address of the blob          xd : this lane's B source per step class (digits or zeros)
 //   xg   : shared address of the blob's group sums / scales
+//   tsel : 0 = both 16-row tiles of the blob, 1 = tile 0 only, 2 = tile 1 only (the other tile's sums stay 0)
 template <int VARIANT>
-__device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane, float (&tot)[kBlobTiles][2])
+__device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane, int tsel,
+                                             float (&tot)[kBlobTiles][2])
 {
     // a nested child reads the parent's top bits; the dropped bits are filled with their mid-point, which
     // is the same as lowering every zero point by that amount
@@ -212,6 +214,7 @@ __device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)
             const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
             static_for<0, kBlobTiles>([&](auto TLI) {
                 constexpr int tile = decltype(TLI)::value;
+                if (tsel == 2 - tile) return;                    // (warp-uniform) this tile belongs to another item
                 const uint4 mw = lds128<(ss * kBlobTiles + tile) * 128>(mbase);
                 int v[2][2];
                 FieldLoop<VARIANT, 0, 0, ss, tile>::run(fbase, bx, c, m1, v);
@@ -228,7 +231,7 @@ __device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)
             const float sc[2] = {__uint_as_float(sc2.x), __uint_as_float(sc2.y)};
             float tt[kBlobTiles][2] = {{tot[0][0], tot[0][1]}, {tot[1][0], tot[1][1]}};
 #pragma unroll 1
-            for (int tile = 0; tile < kBlobTiles; tile++) {
+            for (int tile = tsel == 2 ? 1 : 0; tile < (tsel == 1 ? 1 : kBlobTiles); tile++) {
                 const int st = ss * kBlobTiles + tile;
                 const uint4 mw = lds128(mbase + st * 128);
                 int v[2][2];
@@ -244,10 +247,10 @@ __device__ __forceinline__ void blob_compute(uint32_t blob, const uint32_t (&xd)
 }
 
 // Selects the specialised loop of a variant (variant_index in fq_layout.cuh).
-__device__ __forceinline__ void blob_dispatch(int variant, uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane,
+__device__ __forceinline__ void blob_dispatch(int variant, uint32_t blob, const uint32_t (&xd)[4], uint32_t xg, int lane, int tsel,
                                               float (&tot)[kBlobTiles][2])
 {
-#define FQ_VARIANT_CASE(V) case V: blob_compute<V>(blob, xd, xg, lane, tot); break;
+#define FQ_VARIANT_CASE(V) case V: blob_compute<V>(blob, xd, xg, lane, tsel, tot); break;
     switch (variant) {
         FQ_VARIANT_CASE(0) FQ_VARIANT_CASE(1) FQ_VARIANT_CASE(2) FQ_VARIANT_CASE(3) FQ_VARIANT_CASE(4)
         FQ_VARIANT_CASE(5) FQ_VARIANT_CASE(6) FQ_VARIANT_CASE(7) FQ_VARIANT_CASE(8) FQ_VARIANT_CASE(9)

@@ -51,6 +51,7 @@ struct GemvOp {
     int phase;                   // -1: no ordering
     int n_units;                 // n_chunks * n_rp
     int rot;                     // rotation of the CTA blocks for this op (evens out remainders)
+    int split;                   // batch 1: consumer items per blob: 1 (both 16-row tiles) or 2 (one tile each)
 };
 static_assert(offsetof(GemvOp, blob_read) == 16 && offsetof(GemvOp, partial) == 8, "consumer block of the op descriptor");
 
