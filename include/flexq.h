@@ -254,8 +254,12 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host,
  *   ldx and ldy multiples of 8, 1 <= M <= 2^20.
  * One fused kernel: X tiles arrive by TMA, the stored blobs are dequantised inside the kernel
  * (w^ = (q - z) * s exactly in fp32, rounded once to bf16) into the shared-memory operand tiles of
- * the tensor cores (tcgen05, fp32 accumulation in TMEM), Y is rounded once to bf16.  No workspace,
- * no allocation; enqueues one kernel on `stream` and encodes one tensor map on the host. */
+ * the tensor cores (tcgen05, fp32 accumulation in TMEM), Y is rounded once to bf16.  Enqueues one
+ * kernel on `stream` and encodes one tensor map on the host.  Shapes whose 256 x 256 output tiles would
+ * leave the last wave of thread blocks mostly empty are cut into equal runs of (tile, K stage) work
+ * instead; a tile shared by two blocks is then the fp32 sum of two partial accumulations (summation
+ * order differs from the whole-tile case in the last bit), passed through a 38 MB workspace that the
+ * context allocates the first time such a shape is used.  One fq_gemm at a time per context. */
 int fq_gemm(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int ldx,
             uint16_t* Y_dev, int ldy, void* stream);
 

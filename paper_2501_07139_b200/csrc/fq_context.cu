@@ -197,6 +197,7 @@ int fq_destroy(fq_ctx* ctx)
             if (ctx->stage_done[i]) cudaEventDestroy(ctx->stage_done[i]);
         }
         if (ctx->gemm_ws) cudaFree(ctx->gemm_ws);
+        if (ctx->fused_ws) cudaFree(ctx->fused_ws);
         for (void* p : ctx->owned) cudaFree(p);
         for (Layer& L : ctx->layers)
             for (Variant& v : L.var)
@@ -814,9 +815,26 @@ static int gemm_common(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int
     if (!guard.ok) return FQ_ERR_CUDA;
     const int zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
     const int stride = blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits);
-    if (fused)
+    if (fused) {
+        float* parts = nullptr;
+        unsigned* flags = nullptr;
+        if (gemm_fused_wants_balance(M, L.n_out, ctx->sm_count)) {
+            // partial-sum slots of the tiles that two CTAs share: [flags 4 x (SMs + 1), padded][slot x (SMs + 1)];
+            // allocated the first time a shape asks for balanced runs
+            const size_t flag_bytes = (size_t)round_up((int64_t)((ctx->sm_count + 1) * 4 * sizeof(unsigned)), 256);
+            if (!ctx->fused_ws) {
+                const size_t bytes = flag_bytes + (size_t)(ctx->sm_count + 1) * gemm_fused_part_bytes();
+                FQ_CUDA_OK(cudaMalloc(&ctx->fused_ws, bytes));
+                FQ_CUDA_OK(cudaMemset(ctx->fused_ws, 0, flag_bytes));
+                ctx->fused_epoch = 0;
+            }
+            if (++ctx->fused_epoch == 0) ctx->fused_epoch = 1;               // (0 is the cleared flag)
+            flags = reinterpret_cast<unsigned*>(ctx->fused_ws);
+            parts = reinterpret_cast<float*>(ctx->fused_ws + flag_bytes);
+        }
         return launch_gemm_fused(ctx, v->store, stride, active_fields(L, bits), zero_adjust, L.n_out, L.k_in, X_dev, M, ldx,
-                                 Y_dev, ldy, (cudaStream_t)stream);
+                                 Y_dev, ldy, parts, flags, ctx->fused_epoch, (cudaStream_t)stream);
+    }
     const size_t need = (size_t)L.n_out * L.k_in * 2;
     if (need > ctx->gemm_ws_bytes) {
         FQ_CUDA_OK(cudaDeviceSynchronize());

@@ -20,6 +20,7 @@
 #include <cuda_fp16.h>
 
 #include "fq_internal.cuh"
+#include "fq_ptx.cuh"
 #include "fq_umma.cuh"
 
 namespace fq {
@@ -55,6 +56,49 @@ struct FusedArgs {
     int M, N, K, ldy;
     __nv_bfloat16* Y;
     int* status;
+    // balanced runs (below): one 256 x 256 fp32 slot per CTA, a flag per slot and epilogue warp, the launch number
+    int balanced;
+    float* parts;
+    unsigned* part_flags;
+    unsigned epoch;
+};
+
+constexpr int kPartFloats = kFM * kFN;
+
+// Work of one CTA.  Normally whole tiles, CTA c takes tiles c, c + grid, ...  When that would leave most SMs idle in
+// the last wave (160 tiles on 148 SMs), the host asks for BALANCED RUNS instead: the (tile, K stage) pairs,
+// tile-major, are cut into gridDim.x equal contiguous runs.  A run is at least one tile long (grid <= tiles), hence
+// covers: the rest of a tile that the previous CTA began (ks0 > 0), whole tiles, and the beginning of a tile that the
+// next CTA finishes (ks1 < k_steps).  The CTA that computes the rest does so FIRST and leaves fp32 partial sums in
+// its slot; the CTA that computes the beginning does so LAST, adds the slot and writes the outputs.
+struct WorkItem { int tile, ks0, ks1; };
+struct WorkRun {
+    long long u, u_hi;
+    int k_steps, n_tiles, next_tile;
+    bool balanced;
+    __device__ WorkRun(int n_tiles_, int k_steps_, bool balanced_) : k_steps(k_steps_), n_tiles(n_tiles_), balanced(balanced_)
+    {
+        const long long total = (long long)n_tiles_ * k_steps_;
+        u = total * blockIdx.x / gridDim.x;
+        u_hi = total * (blockIdx.x + 1) / gridDim.x;
+        next_tile = blockIdx.x;
+    }
+    __device__ bool next(WorkItem& it)
+    {
+        if (!balanced) {
+            if (next_tile >= n_tiles) return false;
+            it.tile = next_tile; it.ks0 = 0; it.ks1 = k_steps;
+            next_tile += gridDim.x;
+            return true;
+        }
+        if (u >= u_hi) return false;
+        it.tile = (int)(u / k_steps);
+        it.ks0 = (int)(u % k_steps);
+        const long long left = u_hi - u;
+        it.ks1 = left < k_steps - it.ks0 ? it.ks0 + (int)left : k_steps;
+        u += it.ks1 - it.ks0;
+        return true;
+    }
 };
 
 // Loop whose index is a compile-time constant in the body.
@@ -204,9 +248,11 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
             int stage = 0;
             uint32_t wraps = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int mb = t % m_blocks;                               // m fastest: the blobs of a row block stay in L2
-                for (int ks = 0; ks < k_steps; ks++) {
+            WorkRun run(n_tiles, k_steps, a.balanced != 0);
+            WorkItem it;
+            while (ok && run.next(it)) {
+                const int mb = it.tile % m_blocks;                         // m fastest: the blobs of a row block stay in L2
+                for (int ks = it.ks0; ks < it.ks1; ks++) {
                     if (wraps > 0 && !g_wait(empty0 + 8 * stage, (wraps - 1u) & 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full = full0 + 8 * stage;
                     const uint32_t a_dst = g_smem_u32(smem + stage * FusedSmem::kStageBytes);
@@ -231,11 +277,13 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
             uint32_t wraps = 0;
             int local = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, local++) {
-                // both accumulators belong to this tile: wait until the epilogue has drained the previous one
+            WorkRun run(n_tiles, k_steps, a.balanced != 0);
+            WorkItem it;
+            for (; ok && run.next(it); local++) {
+                // both accumulators belong to this item: wait until the epilogue has drained the previous one
                 if (local > 0 && !g_wait(tempty, (uint32_t)(local - 1) & 1u, abort_flag)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                for (int ks = 0; ks < k_steps; ks++) {
+                for (int ks = it.ks0; ks < it.ks1; ks++) {
                     if (!g_wait(full0 + 8 * stage, wraps & 1u, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = g_smem_u32(smem + stage * FusedSmem::kStageBytes);
@@ -246,7 +294,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                         for (int kk = 0; kk < kFK / 16; kk++) {
                             const uint64_t adesc = umma_desc_sw128(a_addr + h * (FusedSmem::kABytes / 2) + kk * 32);
                             const uint64_t bdesc = umma_desc_sw128(b_addr + kk * 32);
-                            const uint32_t accumulate = (ks > 0 || kk > 0) ? 1u : 0u;
+                            const uint32_t accumulate = (ks > it.ks0 || kk > 0) ? 1u : 0u;
                             asm volatile(
                                 "{\n\t.reg .pred p;\n\t"
                                 "setp.ne.b32 p, %4, 0;\n\t"
@@ -268,14 +316,83 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
         const int quarter = warp & 3;                                   // TMEM lanes 32*quarter .. +31 belong to this warp
         int local = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, local++) {
-            const int mb = t % m_blocks, nb = t / m_blocks;
+        WorkRun run(n_tiles, k_steps, a.balanced != 0);
+        WorkItem it;
+        for (; ok && run.next(it); local++) {
+            const int mb = it.tile % m_blocks, nb = it.tile / m_blocks;
+            const bool dump = it.ks0 > 0;                               // the rest of a tile another CTA began: leave partial sums
+            const bool merge = it.ks1 < k_steps;                        // the beginning of a tile: add the next CTA's partial sums
+            // slot layout: float4 number q (columns 4q .. 4q + 3) of token half h: [h][q][quarter][lane] -- a warp's accesses are contiguous
+            const float4* slot_in = reinterpret_cast<const float4*>(a.parts + (long long)(blockIdx.x + 1) * kPartFloats) + quarter * 32 + lane;
+            float4* slot_out = reinterpret_cast<float4*>(a.parts + (long long)blockIdx.x * kPartFloats) + quarter * 32 + lane;
+            if (merge) {
+                // that CTA computed its part first of all, long ago; the wait is bounded all the same
+                const unsigned* flag = a.part_flags + (blockIdx.x + 1) * 4 + quarter;
+                bool seen = ld_acquire_u32(flag) == a.epoch;
+                if (!seen) {
+                    const unsigned long long t0 = g_ns();
+                    while (!(seen = ld_acquire_u32(flag) == a.epoch) && !*abort_flag && g_ns() - t0 <= kGemmWaitNs) __nanosleep(64);
+                }
+                if (!__all_sync(0xffffffffu, seen)) { ok = false; break; }
+            }
             if (!g_wait<256>(tfull, (uint32_t)local & 1u, abort_flag)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
             for (int h = 0; h < 2; h++) {
                 const int row = mb * kFM + h * 128 + quarter * 32 + lane;    // token
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * kFN);
+                if (merge) {
+                    // 16 columns at a time; the partial sums of the next 16 travel while these are added and stored
+                    float4 p[4], pn[4];
+#pragma unroll
+                    for (int e = 0; e < 4; e++) p[e] = __ldcg(slot_in + ((h * 64 + e) * 4) * 32);
+#pragma unroll 1
+                    for (int cb = 0; cb < kFN / 16; cb++) {
+                        uint32_t v[16];
+                        asm volatile(
+                            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                              "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                            : "r"(taddr0 + (uint32_t)(cb * 16)) : "memory");
+                        if (cb + 1 < kFN / 16) {
+#pragma unroll
+                            for (int e = 0; e < 4; e++) pn[e] = __ldcg(slot_in + ((h * 64 + (cb + 1) * 4 + e) * 4) * 32);
+                        }
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        float f[16];
+#pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            f[4 * e] = __uint_as_float(v[4 * e]) + p[e].x;
+                            f[4 * e + 1] = __uint_as_float(v[4 * e + 1]) + p[e].y;
+                            f[4 * e + 2] = __uint_as_float(v[4 * e + 2]) + p[e].z;
+                            f[4 * e + 3] = __uint_as_float(v[4 * e + 3]) + p[e].w;
+                            p[e] = pn[e];
+                        }
+                        const int col0 = nb * kFN + cb * 16;
+                        if (row < a.M && col0 < a.N) {
+                            __nv_bfloat16* dst = a.Y + (long long)row * a.ldy + col0;
+                            if (col0 + 16 <= a.N) {
+#pragma unroll
+                                for (int q = 0; q < 2; q++) {
+                                    uint4 o;
+                                    uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                                    for (int e = 0; e < 4; e++) {
+                                        const __nv_bfloat162 hh = __floats2bfloat162_rn(f[8 * q + 2 * e], f[8 * q + 2 * e + 1]);
+                                        ow[e] = *reinterpret_cast<const uint32_t*>(&hh);
+                                    }
+                                    *reinterpret_cast<uint4*>(dst + 8 * q) = o;
+                                }
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 16; e++)
+                                    if (col0 + e < a.N) dst[e] = __float2bfloat16_rn(f[e]);
+                            }
+                        }
+                    }
+                    continue;
+                }
 #pragma unroll 1
                 for (int cb = 0; cb < kFN / 32; cb++) {
                     uint32_t v[32];
@@ -289,6 +406,13 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                         : "r"(taddr0 + (uint32_t)(cb * 32)) : "memory");
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (dump) {
+#pragma unroll
+                        for (int e = 0; e < 8; e++)
+                            slot_out[((h * 64 + cb * 8 + e) * 4) * 32] = make_float4(__uint_as_float(v[4 * e]), __uint_as_float(v[4 * e + 1]),
+                                                                                     __uint_as_float(v[4 * e + 2]), __uint_as_float(v[4 * e + 3]));
+                        continue;
+                    }
                     const int col0 = nb * kFN + cb * 32;
                     if (row < a.M && col0 < a.N) {
                         __nv_bfloat16* dst = a.Y + (long long)row * a.ldy + col0;
@@ -313,6 +437,11 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                     }
                 }
             }
+            if (dump) {                                                  // publish this warp's quarter of the slot
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) st_release_u32(a.part_flags + blockIdx.x * 4 + quarter, a.epoch);
+            }
             // the accumulators may be overwritten
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -334,12 +463,14 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
         const uint32_t btile0 = g_smem_u32(smem) + FusedSmem::kABytes;
         long long seq = 0;                                              // stages of this CTA so far, over all its tiles
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-            const int nb = t / m_blocks;
+        WorkRun run(n_tiles, k_steps, a.balanced != 0);
+        WorkItem it;
+        while (ok && run.next(it)) {
+            const int nb = it.tile / m_blocks;
             const int rp = nb * kDqWarps + dw;
             const bool have = rp < n_rp;
             const uint8_t* row_blobs = a.store + (long long)(have ? rp : 0) * a.n_kb * a.blob_stride + lane * 16;
-            for (int ks = 0; ks < k_steps; ks++, seq++) {
+            for (int ks = it.ks0; ks < it.ks1; ks++, seq++) {
                 if ((int)(seq % kDqGroups) != grp_id) continue;
                 const int stage = (int)(seq % kFStages);
                 const uint32_t wraps = (uint32_t)(seq / kFStages);
@@ -425,8 +556,20 @@ bool same_fields(const FieldList& x, const FieldList& y)
 
 }  // namespace
 
+size_t gemm_fused_part_bytes() { return (size_t)kPartFloats * sizeof(float); }
+
+// Balanced runs pay two extra epilogues per CTA; they are worth it when whole tiles would leave the last wave mostly empty.
+bool gemm_fused_wants_balance(int M, int n_out, int sm_count)
+{
+    const long long tiles = (long long)((M + kFM - 1) / kFM) * ((n_out + kFN - 1) / kFN);
+    if (tiles <= sm_count) return false;
+    const long long waves = (tiles + sm_count - 1) / sm_count;
+    return (double)tiles / (double)(waves * sm_count) < 0.80;
+}
+
 int launch_gemm_fused(Ctx* ctx, const void* store, int blob_stride, const FieldList& fl, int zero_adjust, int n_out, int k_in,
-                      const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, cudaStream_t st)
+                      const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, float* parts, unsigned* part_flags, unsigned epoch,
+                      cudaStream_t st)
 {
     CUtensorMap map_x;
     const int rc = make_map(&map_x, X, M, k_in, ldx, 128);
@@ -439,6 +582,7 @@ int launch_gemm_fused(Ctx* ctx, const void* store, int blob_stride, const FieldL
     a.store = static_cast<const uint8_t*>(store); a.n_kb = k_blobs(k_in); a.blob_stride = blob_stride;
     a.zero_adjust = zero_adjust; a.M = M; a.N = n_out; a.K = k_in; a.ldy = ldy;
     a.Y = reinterpret_cast<__nv_bfloat16*>(Y); a.status = ctx->status_dev;
+    a.balanced = parts != nullptr ? 1 : 0; a.parts = parts; a.part_flags = part_flags; a.epoch = epoch;
     const int tiles = ((M + kFM - 1) / kFM) * ((n_out + kFN - 1) / kFN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     switch (variant) {

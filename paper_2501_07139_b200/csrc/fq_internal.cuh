@@ -75,6 +75,8 @@ struct Ctx {
     // prefill: dequantised bf16 copy of the layer being multiplied
     char* gemm_ws = nullptr;
     size_t gemm_ws_bytes = 0;
+    char* fused_ws = nullptr;            // fused GEMM, balanced runs: flags, then one fp32 tile slot per SM (+ 1)
+    unsigned fused_epoch = 0;
     std::vector<void*> owned;    // device buffers allocated by fq_load, freed by fq_destroy
     uint64_t config_epoch = 0;
     unsigned launch_epoch = 0;   // tag of the split-K partials of the latest decode launch (never 0)
@@ -127,7 +129,10 @@ int gemv_chunk_blobs(int bits, int batch);
 size_t gemv_partial_bytes_per_unit(int batch);
 int launch_gemv_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                 // batch 2..8
 int launch_gemm_fused(Ctx* ctx, const void* store, int blob_stride, const FieldList& fl, int zero_adjust, int n_out, int k_in,
-                      const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, cudaStream_t st);
+                      const uint16_t* X, int M, int ldx, uint16_t* Y, int ldy, float* parts, unsigned* part_flags, unsigned epoch,
+                      cudaStream_t st);                   // parts == nullptr: whole tiles; else balanced runs through these slots
+size_t gemm_fused_part_bytes();          // bytes of one CTA's partial-sum slot
+bool gemm_fused_wants_balance(int M, int n_out, int sm_count);
 struct CtaWork;
 int launch_gemv1_single(Ctx* ctx, const GemvOp& op, cudaStream_t st);                // batch 1
 // table_dev: [GemvOp x n_ops][int phase_total x max(n_phases,1)][uint2 strips x sm_count x n_ops]
