@@ -323,10 +323,15 @@ def config_report(P, device, steps, brief=False):
             def pf():
                 for i, sh in enumerate(shapes):
                     fq.fq_gemm(i, xb[sh.k_in], yb[sh.n_out])
+            def pf_two():
+                for i, sh in enumerate(shapes):
+                    fq.fq_gemm_two_pass(i, xb[sh.k_in], yb[sh.n_out])
             ms = _time_ms(pf, max(1, steps // 4), 2)
+            ms_two = _time_ms(pf_two, max(1, steps // 4), 2)
             flop = sum(2.0 * m * sh.n_out * sh.k_in for sh in shapes)
             entry["prefill"] = {"tokens": m, "average_bits": S.average_bits(bits, shapes), "ms_per_pass": ms,
-                                "tflops": flop / ms / 1e9, "frac_of_measured_sustained_bf16": flop / ms / 1e9 / peaks["bf16_tflops_sustained"]}
+                                "tflops": flop / ms / 1e9, "frac_of_measured_sustained_bf16": flop / ms / 1e9 / peaks["bf16_tflops_sustained"],
+                                "two_pass": {"ms_per_pass": ms_two, "tflops": flop / ms_two / 1e9}}
         if fq.fq_status() != 0:
             raise RuntimeError("device status after config report")
         out.append(entry)
