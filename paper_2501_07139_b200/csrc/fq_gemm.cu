@@ -15,6 +15,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "fq_dequant.cuh"
 #include "fq_internal.cuh"
 #include "fq_umma.cuh"
 
@@ -25,86 +26,73 @@ namespace fq {
 // ------------------------------------------------------------------------------- dequantise to bf16
 struct DequantArgs {
     const uint8_t* store;
-    FieldList fl;
     int n_out, k_in, n_kb, blob_stride;
     int zero_adjust;
     __nv_bfloat16* out;              // [n_out][k_in]
 };
 
-// One warp per (row tile, superstep): 16 rows x 256 columns.  The lanes read the stored words exactly as
-// the decode kernel does (coalesced 16-byte chunks), rebuild the codes four at a time (one byte each) and
-// write 8-byte runs of bf16.
-template <int F>
-__device__ __forceinline__ void gather_field(const uint8_t* tile_base, int lane, int shift, uint32_t (&code)[32])
-{
-    constexpr int P = 8 / F;
-    constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
-#pragma unroll
-    for (int jb = 0; jb < F; jb++) {
-        const uint4 w = __ldg(reinterpret_cast<const uint4*>(tile_base + jb * 512 + lane * 16));
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int t = 0; t < P; t++)
-#pragma unroll
-            for (int r = 0; r < 4; r++) code[(P * jb + t) * 4 + r] |= ((ww[r] >> (t * F)) & kMask) << shift;
-    }
-}
-
+// One warp per (row strip of 32, 64 columns): the lanes read the stored words of the two k32 steps exactly as
+// the decode kernel does (16 bytes per lane and field chunk), merge the fields into four codes per register,
+// convert (w^ = (q - z) * s exactly, one rounding to bf16) and write 8-byte runs; the four lanes of a quad
+// cover 32 contiguous bytes of a row.  Specialised per field list like the fused kernel, whose helpers it shares.
+template <int VARIANT>
 __global__ void __launch_bounds__(256) dequant_kernel(const DequantArgs a)
 {
+    constexpr FieldList FL = variant_fields(VARIANT);
+    constexpr int kLoads = fields_loads(FL, FL.n);
+    constexpr bool kSmallCodes = VARIANT < 6;            // PACKED 2..7 bits: codes below 128, no zero adjustment
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
-    const int n_rt = row_tiles(a.n_out), n_ss = supersteps(a.k_in);
-    const long long total = (long long)n_rt * n_ss;
+    const int n_rp = row_pairs(a.n_out), n_st = a.k_in / 64;
+    const long long total = (long long)n_rp * n_st;
     const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
     for (long long ti = warp0; ti < total; ti += n_warps) {
-        const int rt = (int)(ti / n_ss), ss = (int)(ti % n_ss);
-        const int tile = rt % kBlobTiles, ssl = ss % kBlobSteps;
-        const uint8_t* blob = a.store + ((long long)(rt / kBlobTiles) * a.n_kb + ss / kBlobSteps) * a.blob_stride;
-        uint32_t code[32];                               // register (k32 step j, a0..a3): four codes, one per byte
+        const int rp = (int)(ti / n_st), ks = (int)(ti % n_st);       // consecutive warps: consecutive columns of a strip
+        const int kb = ks >> 3, ssl = (ks >> 2) & 1, j0 = (ks & 3) * 2, grp = (ks >> 1) & 1;
+        const uint8_t* blob_lane = a.store + ((long long)rp * a.n_kb + kb) * a.blob_stride + lane * 16;
+        uint4 raw[kBlobTiles][kLoads];
+        uint2 meta[kBlobTiles];
+        load_stage_words<VARIANT, 0>(blob_lane, ssl, j0, raw[0]);
+        load_stage_words<VARIANT, 1>(blob_lane, ssl, j0, raw[1]);
 #pragma unroll
-        for (int i = 0; i < 32; i++) code[i] = 0u;
-        int prefix = 0;
-        for (int fi = 0; fi < a.fl.n; fi++) {
-            const int f = a.fl.width[fi];
-            const uint8_t* tb = blob + blob_field_off(prefix, f, ssl, tile);
-            switch (f) {
-                case 8: gather_field<8>(tb, lane, a.fl.shift[fi], code); break;
-                case 4: gather_field<4>(tb, lane, a.fl.shift[fi], code); break;
-                case 2: gather_field<2>(tb, lane, a.fl.shift[fi], code); break;
-                default: gather_field<1>(tb, lane, a.fl.shift[fi], code); break;
-            }
-            prefix += f;
-        }
-        const uint32_t* meta = reinterpret_cast<const uint32_t*>(blob + blob_meta_off(ssl, tile));
-        float sc[2][2], zp[2][2];                        // [group][row g / g+8]
+        for (int tl = 0; tl < kBlobTiles; tl++)
+            meta[tl] = __ldg(reinterpret_cast<const uint2*>(blob_lane - lane * 16 + blob_meta_off(ssl, tl) + blob_meta_word(grp, g)));
 #pragma unroll
-        for (int grp = 0; grp < 2; grp++)
+        for (int tl = 0; tl < kBlobTiles; tl++) {
+            uint32_t code[2][4];
+            merge_codes<VARIANT>(raw[tl], j0, code);
+            const uint32_t mm[2] = {meta[tl].x, meta[tl].y};
 #pragma unroll
             for (int hr = 0; hr < 2; hr++) {
-                const uint32_t m = __ldg(meta + blob_meta_word(grp, g + 8 * hr) / 4);
-                sc[grp][hr] = __half2float(__ushort_as_half((unsigned short)(m & 0xffffu)));
-                zp[grp][hr] = (float)((int)(m >> 16) - a.zero_adjust);
-            }
+                const long long n = (long long)rp * 32 + tl * kTileRows + g + 8 * hr;
+                if (n >= a.n_out) continue;
+                const float s = __half2float(__ushort_as_half((unsigned short)(mm[hr] & 0xffffu)));
+                const __half2 zz = __half2half2(__int2half_rn(1024 + (int)(mm[hr] >> 16) - a.zero_adjust));
+                const float cc = -(float)(128 + (int)(mm[hr] >> 16)) * s;
+                __nv_bfloat16* row = a.out + n * a.k_in + ks * 64 + 4 * c;
 #pragma unroll
-        for (int j = 0; j < 8; j++)
+                for (int jj = 0; jj < 2; jj++)
 #pragma unroll
-            for (int r = 0; r < 4; r++) {
-                const int hr = r & 1, half = r >> 1;
-                const long long n = (long long)rt * kTileRows + g + 8 * hr;
-                const int k = ss * kStepCols + 32 * j + 16 * half + 4 * c;
-                if (n >= a.n_out || k >= a.k_in) continue;
-                const uint32_t q4 = code[j * 4 + r];
-                const float s = sc[j >> 2][hr], z = zp[j >> 2][hr];
-                const __nv_bfloat162 lo = __floats2bfloat162_rn(((float)(q4 & 0xffu) - z) * s, ((float)((q4 >> 8) & 0xffu) - z) * s);
-                const __nv_bfloat162 hi = __floats2bfloat162_rn(((float)((q4 >> 16) & 0xffu) - z) * s, ((float)(q4 >> 24) - z) * s);
-                uint2 o;
-                o.x = *reinterpret_cast<const uint32_t*>(&lo);
-                o.y = *reinterpret_cast<const uint32_t*>(&hi);
-                *reinterpret_cast<uint2*>(a.out + n * a.k_in + k) = o;
+                    for (int half = 0; half < 2; half++) {
+                        const uint32_t q4 = code[jj][2 * half + hr];          // A register r = 2 * half + row half
+                        const uint2 o = kSmallCodes ? small_codes_to_bf16(q4, cc, s) : codes_to_bf16(q4, zz, s);
+                        *reinterpret_cast<uint2*>(row + 32 * jj + 16 * half) = o;
+                    }
             }
+        }
     }
+}
+
+template <int VARIANT>
+static int launch_dequant(const DequantArgs& da, int sm_count, cudaStream_t st)
+{
+    const long long items = (long long)row_pairs(da.n_out) * (da.k_in / 64);     // one warp each
+    long long blocks = (items + 7) / 8;
+    if (blocks > (long long)sm_count * 8) blocks = (long long)sm_count * 8;
+    dequant_kernel<VARIANT><<<(unsigned)blocks, 256, 0, st>>>(da);
+    FQ_CUDA_OK(cudaGetLastError());
+    return FQ_OK;
 }
 
 // ------------------------------------------------------------------------------- tcgen05 GEMM
@@ -302,18 +290,22 @@ int launch_gemm(Ctx* ctx, const void* store, int blob_stride, const FieldList& f
 {
     // 1. w^ as bf16 [n_out][k_in]
     DequantArgs da{};
-    da.store = static_cast<const uint8_t*>(store); da.fl = fl; da.n_out = n_out; da.k_in = k_in;
+    da.store = static_cast<const uint8_t*>(store); da.n_out = n_out; da.k_in = k_in;
     da.n_kb = k_blobs(k_in); da.blob_stride = blob_stride; da.zero_adjust = zero_adjust;
     da.out = static_cast<__nv_bfloat16*>(w_scratch);
-    const long long items = (long long)row_tiles(n_out) * supersteps(k_in);     // one warp each
-    long long blocks = (items + 7) / 8;
-    if (blocks > ctx->sm_count * 8) blocks = ctx->sm_count * 8;
-    dequant_kernel<<<(unsigned)blocks, 256, 0, st>>>(da);
-    FQ_CUDA_OK(cudaGetLastError());
+    int rc = FQ_ERR_ARG;
+    switch (variant_of_fields(fl)) {
+#define FQ_CASE(V) case V: rc = launch_dequant<V>(da, ctx->sm_count, st); break;
+        FQ_CASE(0) FQ_CASE(1) FQ_CASE(2) FQ_CASE(3) FQ_CASE(4) FQ_CASE(5) FQ_CASE(6)
+        FQ_CASE(7) FQ_CASE(8) FQ_CASE(9) FQ_CASE(10) FQ_CASE(11) FQ_CASE(12) FQ_CASE(13)
+#undef FQ_CASE
+        default: break;
+    }
+    if (rc != FQ_OK) return rc;
 
     // 2. tcgen05 GEMM
     CUtensorMap map_x, map_w;
-    int rc = make_map(&map_x, X, M, k_in, ldx, kBM);
+    rc = make_map(&map_x, X, M, k_in, ldx, kBM);
     if (rc != FQ_OK) return rc;
     rc = make_map(&map_w, w_scratch, n_out, k_in, k_in, kBN);
     if (rc != FQ_OK) return rc;
