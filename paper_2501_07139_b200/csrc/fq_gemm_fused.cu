@@ -58,6 +58,7 @@ struct FusedArgs {
     __nv_bfloat16* Y;
     int* status;
     // balanced runs (below): one 256 x 256 fp32 slot per CTA, a flag per slot and epilogue warp, the launch number
+    int halves;              // token halves (of 128) per tile: 2, or 1 when 256-token tiles would be too few for the SMs
     int balanced;
     float* parts;
     unsigned* part_flags;
@@ -144,7 +145,9 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_ptr;
 
-    const int m_blocks = (a.M + kFM - 1) / kFM, n_blocks = (a.N + kFN - 1) / kFN;
+    const int halves = a.halves;                          // 128-token halves per tile
+    const int tile_m = 128 * halves;
+    const int m_blocks = (a.M + tile_m - 1) / tile_m, n_blocks = (a.N + kFN - 1) / kFN;
     const int n_tiles = m_blocks * n_blocks;
     const int k_steps = a.K / kFK;
 
@@ -163,12 +166,12 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                     const uint32_t full = full0 + 8 * stage;
                     const uint32_t a_dst = g_smem_u32(smem + stage * FusedSmem::kStageBytes);
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                                 ::"r"(full), "r"(FusedSmem::kABytes) : "memory");
+                                 ::"r"(full), "r"(halves * (FusedSmem::kABytes / 2)) : "memory");
 #pragma unroll
                     for (int h = 0; h < 2; h++)
-                        asm volatile(
+                        if (h < halves) asm volatile(
                             "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                            ::"r"(a_dst + h * (FusedSmem::kABytes / 2)), "l"(&map_x), "r"(ks * kFK), "r"(mb * kFM + h * 128), "r"(full)
+                            ::"r"(a_dst + h * (FusedSmem::kABytes / 2)), "l"(&map_x), "r"(ks * kFK), "r"(mb * tile_m + h * 128), "r"(full)
                             : "memory");
                     if (++stage == kFStages) { stage = 0; wraps++; }
                 }
@@ -198,6 +201,7 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
                     for (int h = 0; h < 2; h++)
 #pragma unroll
                         for (int kk = 0; kk < kFK / 16; kk++) {
+                            if (h >= halves) continue;                     // (tiles of 128 tokens use the first accumulator only)
                             const uint64_t adesc = umma_desc_sw128(a_addr + h * (FusedSmem::kABytes / 2) + kk * 32);
                             const uint64_t bdesc = umma_desc_sw128(b_addr + kk * 32);
                             const uint32_t accumulate = (ks > it.ks0 || kk > 0) ? 1u : 0u;
@@ -244,8 +248,8 @@ gemm_fused_kernel(const __grid_constant__ CUtensorMap map_x, const FusedArgs a)
             if (!g_wait<256>(tfull, (uint32_t)local & 1u, abort_flag)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-            for (int h = 0; h < 2; h++) {
-                const int row = mb * kFM + h * 128 + quarter * 32 + lane;    // token
+            for (int h = 0; h < halves; h++) {
+                const int row = mb * tile_m + h * 128 + quarter * 32 + lane;    // token
                 const uint32_t taddr0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(h * kFN);
                 if (merge) {
                     // 16 columns at a time; the partial sums of the next 16 travel while these are added and stored
@@ -457,8 +461,18 @@ int launch_variant(Ctx* ctx, const CUtensorMap& map_x, const FusedArgs& a, int g
 size_t gemm_fused_part_bytes() { return (size_t)kPartFloats * sizeof(float); }
 
 // Balanced runs pay two extra epilogues per CTA; they are worth it when whole tiles would leave the last wave mostly empty.
+// 256-token tiles make every converted weight serve 256 tokens; when they are so few that twice as many still fit
+// the SMs in one wave, tiles of 128 tokens use twice the SMs for the same work.
+int gemm_fused_halves(int M, int n_out, int sm_count)
+{
+    const long long tiles = (long long)((M + kFM - 1) / kFM) * ((n_out + kFN - 1) / kFN);
+    const long long tiles128 = (long long)((M + 127) / 128) * ((n_out + kFN - 1) / kFN);
+    return (tiles128 > tiles && 2 * tiles <= sm_count) ? 1 : 2;
+}
+
 bool gemm_fused_wants_balance(int M, int n_out, int sm_count)
 {
+    if (gemm_fused_halves(M, n_out, sm_count) == 1) return false;
     const long long tiles = (long long)((M + kFM - 1) / kFM) * ((n_out + kFN - 1) / kFN);
     if (tiles <= sm_count) return false;
     const long long waves = (tiles + sm_count - 1) / sm_count;
@@ -479,7 +493,9 @@ int launch_gemm_fused(Ctx* ctx, const void* store, int blob_stride, const FieldL
     a.zero_adjust = zero_adjust; a.M = M; a.N = n_out; a.K = k_in; a.ldy = ldy;
     a.Y = reinterpret_cast<__nv_bfloat16*>(Y); a.status = ctx->status_dev;
     a.balanced = parts != nullptr ? 1 : 0; a.parts = parts; a.part_flags = part_flags; a.epoch = epoch;
-    const int tiles = ((M + kFM - 1) / kFM) * ((n_out + kFN - 1) / kFN);
+    a.halves = gemm_fused_halves(M, n_out, ctx->sm_count);
+    const int tile_m = 128 * a.halves;
+    const int tiles = ((M + tile_m - 1) / tile_m) * ((n_out + kFN - 1) / kFN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     switch (variant) {
 #define FQ_CASE(V) case V: return launch_variant<V>(ctx, map_x, a, grid, st);
