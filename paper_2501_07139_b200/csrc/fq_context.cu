@@ -72,7 +72,7 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.variant = variant_index(L.fmt == FQ_FMT_PLANES, bits);
     op.store = static_cast<const uint8_t*>(v->store);
     op.blob_stride = blob_bytes(L.fmt == FQ_FMT_PLANES ? 8 : bits);
-    op.blob_read = blob_bytes(bits);
+    op.blob_read = blob_bytes(L.fmt == FQ_FMT_PLANES ? plane_read_bits(bits) : bits);   // a nested child reads whole 2-bit fields
     op.x = x;
     op.y = y;
     op.n_out = L.n_out;
@@ -80,7 +80,8 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.n_ss = supersteps(L.k_in);
     op.n_kb = k_blobs(L.k_in);
     op.n_rp = row_pairs(L.n_out);
-    op.chunk_blobs = batch == 1 ? gemv1_chunk_blobs(op.blob_read) : gemv_chunk_blobs(bits, batch);
+    op.chunk_blobs = batch == 1 ? gemv1_chunk_blobs(op.blob_read)
+                                : gemv_chunk_blobs(L.fmt == FQ_FMT_PLANES ? plane_read_bits(bits) : bits, batch);
     op.n_chunks = (op.n_kb + op.chunk_blobs - 1) / op.chunk_blobs;
     op.batch = batch;
     // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
@@ -618,15 +619,15 @@ int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_de
 // Relative cost of a byte, x64, per variant (0..6 packed 2..8 bits, 7..13 nested 2..8 bits).
 static unsigned deal_weight(int variant)
 {
-    static const unsigned w[kVariants] = {125, 112, 66, 78, 78, 84, 48,        // packed 2..8
-                                          133, 107, 103, 114, 127, 124, 120};  // nested 2..8
+    static const unsigned w[kVariants] = {125, 112, 66, 78, 78, 84, 48,      // packed 2..8
+                                          108, 64, 64, 74, 74, 64, 64};      // nested 2..8 (per byte READ: whole 2-bit fields)
     return variant >= 0 && variant < kVariants ? w[variant] : 64u;
 }
 
 // Time a CTA spends on one blob of an op, in arbitrary units: bytes x the relative cost of a byte of the op's
 // variant.  The 8-bit and 4-bit loops keep up with the CTA's share of HBM; variants with more fields per stored
 // bit are bound by the integer pipe and take longer per byte (per-CTA rates of uniform stacks, all CTAs busy:
-// 8 bits 48.8 GB/s, 4: 46.1, 5: 42.8, 6: 42.5, 7: 39.9, 3: 31.5, 2: 27.7; nested children 27 - 34).  The table
+// 8 bits 48.8 GB/s, 4: 46.1, 5: 42.8, 6: 42.5, 7: 39.9, 3: 31.5, 2: 27.7; nested children 21 - 37 by field count).  The table
 // starts from the inverse rates; the 8-bit entry is lower than that because a CTA that streams 8-bit blobs speeds
 // up when its neighbours are compute-bound and leave it more of the HBM (tuned on the mixed 7B stack: the
 // unordered pass went from 4350 to 5380 GB/s, the ordered one from 1.525 to 1.465 ms).

@@ -57,7 +57,7 @@ __device__ __forceinline__ void merge_codes(const uint4 (&raw)[fields_loads(vari
     unrolled<0, FL.n>([&](auto FI) {
         constexpr int fi = decltype(FI)::value, F = FL.width[fi], P = 8 / F, SH = FL.shift[fi];
         constexpr int base = fields_loads(FL, fi);
-        constexpr uint32_t kM = (((1u << F) - 1u) * 0x01010101u) << SH;
+        constexpr uint32_t kM = (field_keep_mask(F, FL.keep[fi]) * 0x01010101u) << SH;
 #pragma unroll
         for (int jj = 0; jj < 2; jj++) {
             const uint4 w = raw[F == 8 ? base + jj : base];
@@ -112,7 +112,7 @@ inline int variant_of_fields(const FieldList& fl)
     for (int v = 0; v < kVariants; v++) {
         const FieldList c = variant_fields(v);
         bool same = c.n == fl.n;
-        for (int i = 0; same && i < c.n; i++) same = c.width[i] == fl.width[i] && c.shift[i] == fl.shift[i];
+        for (int i = 0; same && i < c.n; i++) same = c.width[i] == fl.width[i] && c.shift[i] == fl.shift[i] && c.keep[i] == fl.keep[i];
         if (same) return v;
     }
     return -1;

@@ -249,12 +249,12 @@ __device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_
 //   MAXB 8 : every register is shifted down to class 0; B columns (2b, 2b+1) carry batch entry
 //            4*pass + b; xa[pass] is this lane's B data
 // With one tile per warp and batch 1 the k32 steps of a group may alternate between FQ_GEMV_NA accumulators.
-template <int F, int SHIFT, bool FIRSTF, int MAXB, int TILES>
+template <int F, int KEEP, int SHIFT, bool FIRSTF, int MAXB, int TILES>
 __device__ __forceinline__ void field_step(uint32_t fa, const uint32_t (&xa)[4], uint32_t xoff, bool two_pass, int c,
                                            int (&v)[TILES][MAXB == 1 ? 1 : 2][2][2])
 {
     constexpr int P = 8 / F;                                   // A registers stacked in one word
-    constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
+    constexpr uint32_t kMask = field_keep_mask(F, KEEP) * 0x01010101u;
     constexpr int NP = MAXB == 1 ? 1 : 2;
     constexpr int NA = (TILES == 1 && MAXB == 1) ? FQ_GEMV_NA : 1;   // accumulators per (tile, pass, group)
     int acc[TILES][NP][2][NA][4];
@@ -343,10 +343,10 @@ struct FieldLoop {
     {
         constexpr FieldList FL = variant_fields(VARIANT);
         if constexpr (FI < FL.n) {
-            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
+            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI], KEEP = FL.keep[FI];
             // field array of width F after fields adding up to PREFIX bits; tile (superstep, row tile) = st_tile
             const uint32_t fa = fbase + kBlobSteps * kBlobTiles * 512 * PREFIX + st_tile * (F * 512);
-            field_step<F, SHIFT, FI == 0, MAXB, TILES>(fa, xa, xoff, two_pass, c, v);
+            field_step<F, KEEP, SHIFT, FI == 0, MAXB, TILES>(fa, xa, xoff, two_pass, c, v);
             FieldLoop<VARIANT, FI + 1, PREFIX + F, MAXB, TILES>::run(fbase, st_tile, xa, xoff, two_pass, c, v);
         }
     }

@@ -94,11 +94,12 @@ __device__ __forceinline__ int opaque_minus_one()
 // per row half r and group the integer  2^SHIFT * sum_k field_k * x_int_k  (this lane's step class) to v.
 //   fa : shared address of this lane's 16-byte chunk in the tile's field array, this superstep
 //   bx : B registers of the superstep: bx[jc] = (b0, b1 of step jc, b0, b1 of step jc + 4)
-template <int F, int SHIFT, bool FIRSTF, int OFF>
+template <int F, int KEEP, int SHIFT, bool FIRSTF, int OFF>
 __device__ __forceinline__ void field_step(uint32_t fa, const uint4 (&bx)[4], int c, int m1, int (&v)[2][2])
 {
     constexpr int P = 8 / F;                                   // A registers stacked in one word
-    constexpr uint32_t kMask = ((1u << F) - 1u) * 0x01010101u;
+    constexpr uint32_t kMask = field_keep_mask(F, KEEP) * 0x01010101u;
+    static_assert(F != 4 || KEEP == 4, "the word-minus-low-nibbles shortcut takes whole 4-bit fields");
     int acc[2][4];
     uint4 w[F < 4 ? F : 4];
     static_for<0, (F < 4 ? F : 4)>([&](auto JB) { w[decltype(JB)::value] = lds128<OFF + decltype(JB)::value * 512>(fa); });
@@ -140,10 +141,10 @@ struct FieldLoop {
     {
         constexpr FieldList FL = variant_fields(VARIANT);
         if constexpr (FI < FL.n) {
-            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
+            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI], KEEP = FL.keep[FI];
             // field array of width F after fields adding up to PREFIX bits; tile (SS, TILE) of it
             constexpr int off = kBlobSteps * kBlobTiles * 512 * PREFIX + (SS * kBlobTiles + TILE) * (F * 512);
-            field_step<F, SHIFT, FI == 0, off>(fbase, bx, c, m1, v);
+            field_step<F, KEEP, SHIFT, FI == 0, off>(fbase, bx, c, m1, v);
             FieldLoop<VARIANT, FI + 1, PREFIX + F, SS, TILE>::run(fbase, bx, c, m1, v);
         }
     }
@@ -157,8 +158,8 @@ struct FieldLoopRt {
     {
         constexpr FieldList FL = variant_fields(VARIANT);
         if constexpr (FI < FL.n) {
-            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI];
-            field_step<F, SHIFT, FI == 0, kBlobSteps * kBlobTiles * 512 * PREFIX>(fbase + st * (F * 512), bx, c, m1, v);
+            constexpr int F = FL.width[FI], SHIFT = FL.shift[FI], KEEP = FL.keep[FI];
+            field_step<F, KEEP, SHIFT, FI == 0, kBlobSteps * kBlobTiles * 512 * PREFIX>(fbase + st * (F * 512), bx, c, m1, v);
             FieldLoopRt<VARIANT, FI + 1, PREFIX + F>::run(fbase, st, bx, c, m1, v);
         }
     }

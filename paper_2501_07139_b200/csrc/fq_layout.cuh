@@ -42,9 +42,14 @@ constexpr int kMaxFields = 7;
 
 struct FieldList {
     int n;
-    uint8_t width[kMaxFields];
-    uint8_t shift[kMaxFields];
+    uint8_t width[kMaxFields];    // stored bits of the field
+    uint8_t shift[kMaxFields];    // position of the field's lowest stored bit inside the code
+    uint8_t keep[kMaxFields];     // bits of the field that count, from its top (= width, except for the last field of a
+                                  // nested child of odd width, whose low bit belongs to the bits the child drops)
 };
+
+// Mask of the bits of a field of width f that count.
+FQ_HDC uint32_t field_keep_mask(int f, int keep) { return ((1u << f) - 1u) & ~((1u << (f - keep)) - 1u); }
 
 // Fields of a PACKED variant of `bits` bits (most significant first).
 FQ_HDC FieldList packed_fields(int bits)
@@ -56,24 +61,30 @@ FQ_HDC FieldList packed_fields(int bits)
             rem -= f;
             fl.width[fl.n] = (uint8_t)f;
             fl.shift[fl.n] = (uint8_t)rem;
+            fl.keep[fl.n] = (uint8_t)f;
             fl.n++;
         }
     return fl;
 }
 
-// Fields of the 8-bit PLANES parent restricted to its `bits` most significant bits.
-// Shifts are in parent code units.
+// Fields of the 8-bit PLANES parent restricted to its `bits` most significant bits.  The parent is stored as four
+// 2-bit fields (bits 7..6, 5..4, 3..2, 1..0), most significant first, so a child of b bits is the first ceil(b / 2)
+// fields of every blob; a child of odd width uses only the upper bit of its last field.  Shifts are in parent
+// code units.
 FQ_HDC FieldList plane_fields(int bits)
 {
     FieldList fl{};
-    fl.width[0] = 2; fl.shift[0] = 6; fl.n = 1;
-    for (int p = 5; p >= 8 - bits; p--) {
-        fl.width[fl.n] = 1;
-        fl.shift[fl.n] = (uint8_t)p;
-        fl.n++;
+    fl.n = (bits + 1) / 2;
+    for (int i = 0; i < fl.n; i++) {
+        fl.width[i] = 2;
+        fl.shift[i] = (uint8_t)(6 - 2 * i);
+        fl.keep[i] = 2;
     }
+    if (bits & 1) fl.keep[fl.n - 1] = 1;
     return fl;
 }
+// Stored bits per weight that a child of `bits` bits reads (whole fields).
+FQ_HDC int plane_read_bits(int bits) { return 2 * ((bits + 1) / 2); }
 
 FQ_HD int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 FQ_HD int row_tiles(int n_out) { return (n_out + kTileRows - 1) / kTileRows; }
