@@ -278,7 +278,7 @@ def config_report(P, device, steps, brief=False):
                              "ms_per_pass": ms, "GBps": fp / ms / 1e6, "frac": fp / ms / 1e6 / peaks["hbm_gbs"],
                              "ms_unordered": ms_free, "GBps_unordered": fp / ms_free / 1e6})
             del xs, ys
-        entry = {"config": cfg, "workload": f"{model}-shaped stack, nested bit-planes, {n_cfg}-configuration chain",
+        entry = {"config": cfg, "workload": f"{model}-shaped stack, nested format (one 8-bit parent per layer), {n_cfg}-configuration chain",
                  "storage_bytes": fq.fq_storage_bytes(), "weight_bytes_moved_by_switches": 0, "decode": rows}
         if steps_freed:
             entry["transitions"] = {"steps": len(steps_freed), "one_way": True, "bytes_loaded_total": int(sum(steps_loaded)),

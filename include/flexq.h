@@ -36,7 +36,7 @@ extern "C" {
 typedef struct fq_ctx fq_ctx;   /* opaque */
 
 enum { FQ_FMT_PACKED = 0,       /* one stored variant per bit-width (Sec. III-A: QM(n) variants)   */
-       FQ_FMT_PLANES = 1 };     /* one 8-bit parent in nested bit-planes (Sec. II-B, AnyPrecision) */
+       FQ_FMT_PLANES = 1 };     /* one 8-bit parent whose bits are nested, most significant first (Sec. II-B, AnyPrecision) */
 
 enum { FQ_OK = 0,
        FQ_ERR_ARG = -1,         /* NULL pointer, bad layer index, bad enum                */
@@ -82,9 +82,10 @@ int fq_quantize_layer(const float* w_dev, int n_out, int k_in, int bits, int gro
  * (Sec. III-A: every module is stored at a few bit-widths; Sec. II-B for PLANES).
  *   PACKED: `bits` in [2,8] is the width of this variant; call again with another width
  *           to add a variant of the same layer (same shape).
- *   PLANES: `bits` must be 8; the parent is stored as a 2-bit top field plus six 1-bit
- *           planes, most significant first inside every blob, so a b-bit child reads exactly
- *           the first b/8 of every blob's codes and every b in [2,8] becomes selectable.
+ *   PLANES: `bits` must be 8; the parent is stored as four 2-bit fields (bits 7..6, 5..4, 3..2,
+ *           1..0), most significant first inside every blob, so a b-bit child reads the first
+ *           ceil(b / 2) fields of every blob (a child of odd width ignores the low bit of its last
+ *           field) and every b in [2,8] becomes selectable.
  *   codes_dev   uint8 [n_out][k_in], one code per byte; read, not retained.
  *   scales_dev, zeros_dev   fp16 [n_out][k_in/128]; read, not retained.
  *   store_out_dev fq_store_bytes() bytes, 256-byte aligned; written and RETAINED.
@@ -276,7 +277,7 @@ int fq_gemm_two_pass(fq_ctx* ctx, int layer, const uint16_t* X_dev, int M, int l
  *   PACKED: uint32 [n_out][k_in*bits/32], per row a little-endian bitstream, code k in bits
  *           [k*bits, (k+1)*bits).
  *   PLANES: uint32 [bits][n_out][k_in/32], plane t holds parent bit 7-t, bit (k%32) of a
- *           word belongs to column k; only the first `bits` stored planes are read.
+ *           word belongs to column k; rebuilt from the first ceil(bits / 2) stored fields.
  * out_dev: n_out*k_in*bits/8 bytes. */
 int fq_export_layer(fq_ctx* ctx, int layer, int bits, void* out_dev, void* stream);
 /* Writes the stored scales and zero points back as fp16 [n_out][k_in/128] each. */

@@ -3,8 +3,8 @@
 // A stored variant is a list of FIELD ARRAYS, most significant field first.  A field is
 // f in {8,4,2,1} consecutive bits of every code, (code >> shift) & (2^f - 1):
 //   PACKED b bits : the binary decomposition of b   (7 -> 4,2,1;  5 -> 4,1;  3 -> 2,1 ...)
-//   PLANES parent : a 2-bit top field (bits 7,6) followed by six 1-bit planes (5 .. 0),
-//                   so a b-bit child is the first b-1 arrays = the first b/8 of the bytes.
+//   PLANES parent : four 2-bit fields (bits 7..6, 5..4, 3..2, 1..0), so a b-bit child is the first
+//                   ceil(b / 2) arrays; a child of odd width ignores the low bit of its last field.
 // Storage is cut into BLOBS: one blob = one row pair (32 rows = two 16-row tiles) x 512 columns
 // (two "supersteps" of 256).  A blob holds, in this order,
 //     scale/zero words   [superstep][tile][row & 7][group][row >> 3]             (512 B)
@@ -13,7 +13,7 @@
 //     field array 1 ...                                                          (most significant first)
 // and blobs are ordered [row_pair][k_blob].  Everything a decode unit needs is therefore ONE
 // contiguous range for a PACKED variant (one bulk copy), and for a nested child the first
-// 512 + 2048*b bytes of every blob (one bulk copy per blob): lower planes are never touched.
+// 512 + 4096 * ceil(b / 2) bytes of every blob (one bulk copy per blob): lower fields are never touched.
 // The order inside a tile is the order in which a warp consumes the values as A-operand
 // registers of the 8-bit mma.m16n8k32 (lane = 4*g + c owns rows g, g+8; in k32 step j it owns
 // columns 32j + 4c .. +3 and 32j + 16 + 4c .. +3).  A 32-bit word holds P = 8/f A-registers

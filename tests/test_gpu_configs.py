@@ -1,4 +1,4 @@
-"""Full-size elastic configurations in the nested bit-plane format (one stored 8-bit parent per layer):
+"""Full-size elastic configurations in the nested format (one stored 8-bit parent per layer, children read its leading bits):
 the 7B-shaped stack with its 12-configuration chain and the 13B-shaped stack with its 16-configuration
 chain.  Footprints are compared bit-for-bit with the oracle, decode / prefill outputs on sampled rows."""
 import time
