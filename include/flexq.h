@@ -201,7 +201,8 @@ int fq_sqdiff(const uint16_t* a_bf16_dev, const uint16_t* b_bf16_dev, size_t n, 
 
 /* Decode (Sec. II-A): y[n] = sum_k x[k] * w^[n][k] at the layer's active bit-width.
  *   x_dev fp16 [k_in], y_dev fp16 [n_out]; both 16-byte aligned.  fp32 accumulation.
- *   k_in <= 14336 (the activations of one 32-row strip stay in shared memory); FQ_ERR_SHAPE otherwise.
+ *   Layers with k_in <= 14336 run in the batch-1 kernel (the activations of one 32-row strip stay in shared
+ *   memory); wider layers run in the batch kernel, slower per byte but without a limit on k_in.
  * Enqueues one kernel on `stream`; neither allocates (the scratch was reserved by fq_pack_layer) nor
  * synchronises.  An activation group that holds an infinity or a NaN makes every output NaN. */
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream);

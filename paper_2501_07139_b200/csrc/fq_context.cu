@@ -50,7 +50,9 @@ constexpr int kSplitBelowBlobsPerCta = 48;
 constexpr int kSplitAboveFields = 2;
 
 // Fills the device descriptor of one decode op (everything except workspace pointers and unit_base).
-int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch, GemvOp& op)
+//   one : the op runs in the batch-1 kernel (gemv1); otherwise in the batch kernel, which also serves batch 1 for
+//         layers whose k_in exceeds what the batch-1 kernel keeps in shared memory
+int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch, bool one, GemvOp& op)
 {
     if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
     const Layer& L = ctx->layers[layer];
@@ -80,28 +82,28 @@ int fill_op(const Ctx* ctx, int layer, const uint16_t* x, uint16_t* y, int batch
     op.n_ss = supersteps(L.k_in);
     op.n_kb = k_blobs(L.k_in);
     op.n_rp = row_pairs(L.n_out);
-    op.chunk_blobs = batch == 1 ? gemv1_chunk_blobs(op.blob_read)
+    op.chunk_blobs = one ? gemv1_chunk_blobs(op.blob_read)
                                 : gemv_chunk_blobs(L.fmt == FQ_FMT_PLANES ? plane_read_bits(bits) : bits, batch);
     op.n_chunks = (op.n_kb + op.chunk_blobs - 1) / op.chunk_blobs;
     op.batch = batch;
     // nested child: codes are the parent's top bits; the dropped bits are filled with their mid-point
     op.zero_adjust = (L.fmt == FQ_FMT_PLANES && bits < 8) ? (1 << (7 - bits)) : 0;
     // what is dealt to the CTAs: batch 1 the blobs of every strip, batch 2..8 the K chunks of every row pair
-    op.n_units = (batch == 1 ? op.n_kb : op.n_chunks) * op.n_rp;
+    op.n_units = (one ? op.n_kb : op.n_chunks) * op.n_rp;
     if ((long long)op.n_units * 1024 >= (1ll << 31)) return FQ_ERR_SHAPE;              // 32-bit unit arithmetic on the device
-    if (batch == 1 && L.k_in > gemv1_max_k()) return FQ_ERR_SHAPE;                   // a strip's activations stay in shared memory
+    if (one && (batch != 1 || L.k_in > gemv1_max_k())) return FQ_ERR_SHAPE;                   // a strip's activations stay in shared memory
     op.phase = -1;
     op.rot = 0;
     // a lone matrix is a few blobs per CTA: items of one 16-row tile spread them over twice as many consumer warps
-    op.split = (batch == 1 && fl.n > kSplitAboveFields && op.n_units < kSplitBelowBlobsPerCta * ctx->sm_count) ? 2 : 1;
+    op.split = (one && fl.n > kSplitAboveFields && op.n_units < kSplitBelowBlobsPerCta * ctx->sm_count) ? 2 : 1;
     return FQ_OK;
 }
 
 // Split-K scratch of one op.  Batch 1: one tagged word per (strip, blob, row) -- only strips that two CTAs
 // share are ever written.  Batch 2..8: one tagged word per (row pair, K chunk, row, batch entry).
-size_t op_partial_bytes(const GemvOp& op, int max_batch)
+size_t op_partial_bytes(const GemvOp& op, bool one, int max_batch)
 {
-    if (max_batch <= 1) return op.n_kb <= 1 ? 0 : (size_t)op.n_rp * op.n_kb * 32 * sizeof(unsigned long long);
+    if (one) return op.n_kb <= 1 ? 0 : (size_t)op.n_rp * op.n_kb * 32 * sizeof(unsigned long long);
     if (op.n_chunks <= 1) return 0;
     return (size_t)op.n_rp * op.n_chunks * gemv_partial_bytes_per_unit(max_batch);
 }
@@ -589,15 +591,17 @@ int fq_gemv_batched(fq_ctx* ctx, int layer, const uint16_t* x_dev, int batch, ui
 {
     if (!ctx) return FQ_ERR_ARG;
     GemvOp op;
-    int rc = fill_op(ctx, layer, x_dev, y_dev, batch, op);
+    if (layer < 0 || layer >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+    const bool one = batch == 1 && ctx->layers[layer].k_in <= gemv1_max_k();     // else the batch kernel (any K)
+    int rc = fill_op(ctx, layer, x_dev, y_dev, batch, one, op);
     if (rc != FQ_OK) return rc;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
-    const size_t pb = op_partial_bytes(op, batch);
+    const size_t pb = op_partial_bytes(op, one, batch);
     rc = ensure_workspace(ctx, kPartialBase + pb + 256);
     if (rc != FQ_OK) return rc;
     op.partial = reinterpret_cast<unsigned long long*>(ctx->ws + kPartialBase);
-    return batch == 1 ? launch_gemv1_single(ctx, op, (cudaStream_t)stream) : launch_gemv_single(ctx, op, (cudaStream_t)stream);
+    return one ? launch_gemv1_single(ctx, op, (cudaStream_t)stream) : launch_gemv_single(ctx, op, (cudaStream_t)stream);
 }
 
 int fq_gemv(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_dev, void* stream)
@@ -609,11 +613,11 @@ int fq_gemv_static(fq_ctx* ctx, int layer, const uint16_t* x_dev, uint16_t* y_de
 {
     if (!ctx) return FQ_ERR_ARG;
     GemvOp op;
-    const int rc = fill_op(ctx, layer, x_dev, y_dev, 1, op);
+    const int rc = fill_op(ctx, layer, x_dev, y_dev, 1, true, op);
     if (rc != FQ_OK) return rc;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
-    return launch_gemv_static(ctx, op, op_partial_bytes(op, 1), (cudaStream_t)stream);
+    return launch_gemv_static(ctx, op, op_partial_bytes(op, true, 1), (cudaStream_t)stream);
 }
 
 // Relative cost of a byte, x64, per variant (0..6 packed 2..8 bits, 7..13 nested 2..8 bits).
@@ -641,13 +645,19 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
 {
     if (!ctx || !layers_host || !x_dev_host || !y_dev_host || n_ops < 1) return FQ_ERR_ARG;
     if (batch < 1 || batch > FQ_MAX_BATCH) return FQ_ERR_SHAPE;
+    // the batch-1 kernel keeps a strip's activations in shared memory: a list with a wider layer runs in the batch kernel
+    bool one = batch == 1;
+    for (int i = 0; i < n_ops && one; i++) {
+        if (layers_host[i] < 0 || layers_host[i] >= (int)ctx->layers.size()) return FQ_ERR_ARG;
+        if (ctx->layers[layers_host[i]].k_in > gemv1_max_k()) one = false;
+    }
     int n_phases = 0;
     if (phases_host) {
         if (phases_host[0] != 0) return FQ_ERR_ARG;
         for (int i = 1; i < n_ops; i++)
             if (phases_host[i] < phases_host[i - 1] || phases_host[i] > phases_host[i - 1] + 1) return FQ_ERR_ARG;
         n_phases = phases_host[n_ops - 1] + 1;
-        if (n_phases > (batch == 1 ? gemv1_max_phases() : kMaxPhases)) return FQ_ERR_SHAPE;
+        if (n_phases > (one ? gemv1_max_phases() : kMaxPhases)) return FQ_ERR_SHAPE;
     }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return FQ_ERR_CUDA;
@@ -669,10 +679,10 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
     // batch 1:    [GemvOp x n_ops][int phase_total x np][uint2 strips x sm_count x n_ops]
     // batch 2..8: [GemvOp x n_ops][long long phase_total x np][int cta_units x sm_count]
     const size_t range_off = (size_t)round_up((int64_t)((size_t)n_ops * sizeof(GemvOp) + (size_t)np * sizeof(int)), 8);
-    const size_t table_bytes = batch == 1 ? range_off + (size_t)ctx->sm_count * n_ops * sizeof(uint2)
+    const size_t table_bytes = one ? range_off + (size_t)ctx->sm_count * n_ops * sizeof(uint2)
                                           : (size_t)n_ops * sizeof(GemvOp) + (size_t)np * sizeof(long long) +
                                                 (size_t)ctx->sm_count * sizeof(int);
-    if (batch == 1 && n_ops > gemv1_max_ops()) return FQ_ERR_SHAPE;
+    if (one && n_ops > gemv1_max_ops()) return FQ_ERR_SHAPE;
 
     if (!(ctx->stack_valid && ctx->stack_sig == sig)) {
         ctx->stack_valid = false;                           // until the new table is complete
@@ -692,23 +702,23 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         long long unit_base = 0;
         std::vector<long long> bases(n_ops);
         for (int i = 0; i < n_ops; i++) {
-            const int rc = fill_op(ctx, layers_host[i], x_dev_host[i], y_dev_host[i], batch, ops[i]);
+            const int rc = fill_op(ctx, layers_host[i], x_dev_host[i], y_dev_host[i], batch, one, ops[i]);
             if (rc != FQ_OK) return rc;
             ops[i].phase = phases_host ? phases_host[i] : -1;
             bases[i] = unit_base;
             unit_base += ops[i].n_units;
-            ws_need += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
+            ws_need += (size_t)round_up((int64_t)op_partial_bytes(ops[i], one, batch), 256);
         }
         const int rc = ensure_workspace(ctx, ws_need + 256);   // (no allocation when every layer appears once)
         if (rc != FQ_OK) return rc;
         size_t poff = kPartialBase;
         for (int i = 0; i < n_ops; i++) {
             ops[i].partial = reinterpret_cast<unsigned long long*>(ctx->ws + poff);
-            poff += (size_t)round_up((int64_t)op_partial_bytes(ops[i], batch), 256);
+            poff += (size_t)round_up((int64_t)op_partial_bytes(ops[i], one, batch), 256);
         }
         const int grid = (int)(unit_base < ctx->sm_count ? unit_base : ctx->sm_count);
         for (int i = 0; i < n_ops; i++) ops[i].rot = (int)(bases[i] % (grid > 0 ? grid : 1));
-        if (batch == 1) {
+        if (one) {
             // per phase: CTAs that finish at least one strip (each reports once when its strips are done)
             int* phase_total = reinterpret_cast<int*>(host + (size_t)n_ops * sizeof(GemvOp));
             for (int p = 0; p < np; p++) phase_total[p] = 0;
@@ -796,7 +806,7 @@ int fq_gemv_stack(fq_ctx* ctx, int n_ops, const int* layers_host, const uint16_t
         ctx->stack_sig.swap(sig);
         ctx->stack_valid = true;
     }
-    return batch == 1 ? launch_gemv1_stack(ctx, ctx->stack_hdr, ctx->stack_dev, st)
+    return one ? launch_gemv1_stack(ctx, ctx->stack_hdr, ctx->stack_dev, st)
                       : launch_gemv_stack(ctx, ctx->stack_hdr, ctx->stack_dev, batch, st);
 }
 

@@ -151,3 +151,40 @@ def test_decode_calls_do_not_allocate(P):
     assert fq.fq_status() == 0
     assert torch.cuda.mem_get_info()[0] == free0
     fq.fq_destroy()
+
+
+@pytest.mark.parametrize("fmt_bits", [(0, 4), (1, 5)])
+def test_layer_wider_than_the_batch1_kernel_holds(P, fmt_bits):
+    """k_in = 16384 is more than the batch-1 kernel keeps in shared memory (14336): fq_gemv and a batch-1
+    fq_gemv_stack then run in the batch kernel; fq_gemv_static, which has no other kernel, refuses."""
+    fmt, bits = fmt_bits
+    n, k = 96, 16384
+    stored = 8 if fmt == 1 else bits
+    codes, s, z = make_layer(160, bits, n, k, stored)
+    fq = P.FlexQ(2)
+    fq.fq_pack_layer(0, *to_dev(codes, s, z), stored, fmt)
+    small = make_layer(160, 9, 64, 512, 4)
+    fq.fq_pack_layer(1, *to_dev(*small), 4, P.FQ_FMT_PACKED)
+    fq.fq_set_config([bits, 4])
+    x = x_fp16(160, bits, 1, k).cuda()[0]
+    y = torch.full((n,), float("nan"), dtype=torch.float16, device="cuda")
+    fq.fq_gemv(0, x, y)
+    assert fq.fq_status() == 0
+    ref = (O.gemv(codes >> (8 - bits), s, z, bits, bits_of(x[None]), parent_bits=8) if fmt == 1
+           else O.gemv(codes, s, z, bits, bits_of(x[None])))[0]
+    got = f64_of(y)
+    assert np.all(np.isfinite(got)) and O.rel_l2(got, ref) <= GEMV_TOL
+    assert np.max(np.abs(got - ref)) <= 4 * GEMV_TOL * np.max(np.abs(ref))
+    # the same layer inside a dependency-ordered batch-1 stack next to a narrow one
+    x1 = x_fp16(160, 7, 1, 512).cuda()[0]
+    ys = [torch.full((n,), float("nan"), dtype=torch.float16, device="cuda"),
+          torch.full((64,), float("nan"), dtype=torch.float16, device="cuda")]
+    fq.fq_gemv_stack([0, 1], [x, x1], ys, [0, 1], 1)
+    assert fq.fq_status() == 0
+    assert O.rel_l2(f64_of(ys[0]), ref) <= GEMV_TOL
+    ref1 = O.gemv(*small, 4, bits_of(x1[None]))[0]
+    assert O.rel_l2(f64_of(ys[1]), ref1) <= GEMV_TOL
+    with pytest.raises(P.FlexQError) as e:
+        fq.fq_gemv_static(0, x, y)
+    assert e.value.code == -3
+    fq.fq_destroy()
